@@ -1,0 +1,141 @@
+"""ctypes front-end of the CPU oracle (oracle/ic_oracle.c).  Test infrastructure only.
+
+The arithmetic lives in the C file; this module only compiles it with gcc,
+marshals numpy arrays and returns numpy arrays.  bf16 data travels as uint16
+bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ic_oracle.c")
+_LIB = os.path.join(_HERE, "libic_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+BF16 = 0
+F32 = 1
+
+
+def build_oracle(force: bool = False) -> str:
+    """Compile the C oracle into oracle/libic_oracle.so (if stale) and return its path."""
+    with _lock:
+        stale = (
+            force
+            or not os.path.exists(_LIB)
+            or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        )
+        if stale:
+            tmp = _LIB + ".tmp.%d" % os.getpid()
+            cmd = [
+                "gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
+                "-ffp-contract=off", "-fno-fast-math", "-Wall", "-Wextra",
+                "-o", tmp, _SRC, "-lm",
+            ]
+            subprocess.run(cmd, check=True)
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build_oracle())
+        lib.ic_oracle_bf16_to_f32.restype = ctypes.c_float
+        lib.ic_oracle_bf16_to_f32.argtypes = [ctypes.c_uint16]
+        lib.ic_oracle_f32_to_bf16.restype = ctypes.c_uint16
+        lib.ic_oracle_f32_to_bf16.argtypes = [ctypes.c_float]
+        lib.ic_oracle_search.restype = ctypes.c_int
+        lib.ic_oracle_search.argtypes = [
+            ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32,
+            ctypes.c_void_p, ctypes.c_int, ctypes.c_int32, ctypes.c_int32, ctypes.c_int,
+            ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+            ctypes.c_void_p,
+        ]
+        _lib = lib
+    return _lib
+
+
+def bf16_bits_to_f32(bits) -> np.ndarray:
+    """Widen bf16 bit patterns (uint16) to fp32, element by element, through the C helper."""
+    lib = _load()
+    b = np.asarray(bits, dtype=np.uint16)
+    out = np.empty(b.shape, dtype=np.float32)
+    flat_in, flat_out = b.reshape(-1), out.reshape(-1)
+    for i in range(flat_in.size):
+        flat_out[i] = lib.ic_oracle_bf16_to_f32(int(flat_in[i]))
+    return out
+
+
+def f32_to_bf16_bits(x) -> np.ndarray:
+    """Round fp32 values to bf16 (nearest, ties to even) through the C helper; returns uint16."""
+    lib = _load()
+    a = np.asarray(x, dtype=np.float32)
+    out = np.empty(a.shape, dtype=np.uint16)
+    flat_in, flat_out = a.reshape(-1), out.reshape(-1)
+    for i in range(flat_in.size):
+        flat_out[i] = lib.ic_oracle_f32_to_bf16(float(flat_in[i]))
+    return out
+
+
+def _as_matrix(a, what: str):
+    a = np.ascontiguousarray(a)
+    if a.dtype == np.uint16:
+        return a, BF16
+    if a.dtype == np.float32:
+        return a, F32
+    raise TypeError(f"{what}: expected float32 values or uint16 bf16 bit patterns, got {a.dtype}")
+
+
+def default_threads() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:  # pragma: no cover
+        return max(1, os.cpu_count() or 1)
+
+
+def search(x, q, k: int, ids=None, normalize: bool = False, round_bf16: bool = False,
+           threads: int | None = None, want_all_scores: bool = False):
+    """Exhaustive cosine/inner-product top-k of every query row against every cache row.
+
+    x: [n, d] float32, or uint16 holding bf16 bits.  q: [nq, d] likewise.
+    ids: optional int64 [n] labels (default: the slot number).
+    round_bf16: round float32 inputs to bf16 first (what a bf16 store keeps).
+    Returns dict(ids [nq,k] int64, scores [nq,k] float32, slots [nq,k] int64,
+    all_scores [nq,n] float32 or None).  Rows past min(k, n) are (-1, -inf, -1).
+    """
+    lib = _load()
+    x, xdt = _as_matrix(x, "x")
+    q, qdt = _as_matrix(q, "q")
+    if x.ndim != 2 or q.ndim != 2:
+        raise ValueError("x and q must be 2-D")
+    n, d = x.shape
+    nq = q.shape[0]
+    if nq and n and q.shape[1] != d:
+        raise ValueError("dimension mismatch")
+    if n == 0:
+        d = q.shape[1]
+    if ids is not None:
+        ids = np.ascontiguousarray(ids, dtype=np.int64)
+        if ids.shape != (n,):
+            raise ValueError("ids must have shape [n]")
+    out_ids = np.empty((nq, k), dtype=np.int64)
+    out_scores = np.empty((nq, k), dtype=np.float32)
+    out_slots = np.empty((nq, k), dtype=np.int64)
+    all_scores = np.empty((nq, n), dtype=np.float32) if want_all_scores else None
+    rc = lib.ic_oracle_search(
+        x.ctypes.data, xdt, ids.ctypes.data if ids is not None else None, n, d,
+        q.ctypes.data, qdt, nq, k, int(bool(normalize)), int(bool(round_bf16)),
+        int(threads or default_threads()),
+        out_ids.ctypes.data, out_scores.ctypes.data, out_slots.ctypes.data,
+        all_scores.ctypes.data if all_scores is not None else None,
+    )
+    if rc != 0:
+        raise RuntimeError(f"ic_oracle_search failed with code {rc}")
+    return {"ids": out_ids, "scores": out_scores, "slots": out_slots, "all_scores": all_scores}
