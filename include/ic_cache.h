@@ -1,0 +1,178 @@
+/*
+ * ic_cache.h - C ABI of the B200 example-retrieval library.
+ *
+ * The library implements stage 1 of IC-Cache's example selection: keep one dense embedding
+ * per cached request and, for each batch of incoming request embeddings, return the k cached
+ * examples with the highest cosine similarity, with their ids and scores (paper Sec. 4.1,
+ * "Two-Stage Scalable Example Selection"; Algorithm 1, RetrieveExamples stage 1,
+ * GetSimilarExamples(request_emb, examples)).  Registration of a served request
+ * (client.update_cache in the client listing of Sec. 3; step 4 of the overview figure) is
+ * ic_cache_insert.
+ *
+ * Storage: a row-major bf16 slab [capacity, dim] in device memory plus an int64 id per row.
+ * Scores are inner products of the stored bf16 rows with the bf16-rounded query, accumulated
+ * in fp32; they equal cosine similarity when inputs are unit vectors or `normalize` is set.
+ *
+ * Conventions common to all calls
+ *   - Unless a call says "host", every data pointer is a DEVICE pointer on the handle's
+ *     device, dense and row-major.  The caller owns those buffers; the library never frees
+ *     or retains them past the work it enqueues.
+ *   - insert/query validate on the host, enqueue kernels on the handle's stream and return
+ *     without synchronising.  Outputs are valid once that stream has reached the call.  A
+ *     query enqueued after an insert on the same stream sees the inserted rows.
+ *   - One handle is bound to one stream and is not thread-safe; handles are independent.
+ *   - Every call returns IC_OK or a negative ic_status.  On a non-OK return nothing was
+ *     enqueued and the cache is unchanged (an insert is all-or-nothing).  The paper's
+ *     fault-tolerance rule (Sec. 5, "Fault Tolerance": bypass the retriever when it fails)
+ *     maps to: treat any non-OK status as "serve without examples".
+ *   - There is no CPU fallback: without a CUDA device ic_cache_create fails.
+ */
+#ifndef IC_CACHE_H_
+#define IC_CACHE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ic_cache ic_cache_t; /* opaque, owned by the library */
+
+enum ic_status {
+  IC_OK = 0,
+  IC_ERR_INVALID = -1,     /* bad argument (NULL pointer, bad dim/k/count, host pointer) */
+  IC_ERR_NOMEM = -2,       /* device allocation failed or caller workspace too small     */
+  IC_ERR_FULL = -3,        /* insert would exceed capacity                                */
+  IC_ERR_CUDA = -4,        /* CUDA runtime/driver error, or no usable device              */
+  IC_ERR_UNSUPPORTED = -5, /* shape outside what the forced kernel path supports          */
+  IC_ERR_TIMEOUT = -6      /* a bounded device-side wait expired in an earlier launch     */
+};
+
+enum ic_dtype { IC_BF16 = 0, IC_F32 = 1 };
+
+/* Kernel path used for scoring (see ic_cache_plan). */
+enum ic_path {
+  IC_PATH_AUTO = 0,    /* chosen from nq: scan for small batches, tensor cores otherwise  */
+  IC_PATH_GENERIC = 1, /* plain CUDA-core kernel, any shape; slow, kept as a cross-check  */
+  IC_PATH_SCAN = 2,    /* bulk-copy staged CUDA-core scan, nq <= 4 per pass, dim <= 1024  */
+  IC_PATH_UMMA = 3     /* tcgen05 tensor-core tiles with the top-k fused in the epilogue  */
+};
+
+#define IC_MAX_K 128        /* largest k accepted by ic_cache_query                         */
+#define IC_MAX_DIM 4096     /* largest embedding dimension; dim must be a multiple of 8     */
+
+/* Options for ic_cache_create_ex.  Zero-initialise, set struct_size = sizeof, then fill. */
+typedef struct ic_cache_opts {
+  uint32_t struct_size; /* sizeof(ic_cache_opts_t) of the caller's build                   */
+  int32_t device;       /* CUDA device ordinal; -1 = the current device                    */
+  int32_t input_dtype;  /* ic_dtype of the emb and q pointers (default IC_BF16)            */
+  int32_t normalize;    /* 1: L2-normalise rows on insert and queries on query (fp32)      */
+  void* slab;           /* optional caller-owned device buffer, capacity*dim*2 bytes,
+                           256-byte aligned; NULL = the library allocates                  */
+  void* ids;            /* optional caller-owned device buffer, capacity*8 bytes           */
+  void* stream;         /* cudaStream_t; NULL = the legacy default stream                  */
+} ic_cache_opts_t;
+
+/* Host-side launch plan for one query call; pure function of its arguments. */
+typedef struct ic_cache_plan {
+  int32_t path;          /* ic_path actually used                                          */
+  int32_t query_tile;    /* queries handled together by one CTA                            */
+  int32_t n_query_tiles; /* per launch                                                     */
+  int32_t n_partitions;  /* row partitions = partial top-k lists per query                 */
+  int32_t n_ctas;        /* CTAs of the scoring kernel                                     */
+  int32_t n_stages;      /* shared-memory ring stages (0 for the generic path)             */
+  int32_t smem_bytes;    /* dynamic shared memory of the scoring kernel                    */
+  int32_t n_launches;    /* scoring launches needed for the whole batch                    */
+} ic_cache_plan_t;
+
+/*
+ * Create an empty cache for embeddings of `dim` components with room for `capacity` entries
+ * on the current device, input dtype bf16, no normalisation, legacy default stream.
+ * dim: multiple of 8, 8 <= dim <= IC_MAX_DIM.  capacity: 1 .. 2^32 - 2.
+ * Returns NULL on failure; ic_cache_last_error() then describes why.
+ */
+ic_cache_t* ic_cache_create(int32_t dim, int64_t capacity);
+
+/* As ic_cache_create, with options (NULL opts = defaults).  Buffers passed in opts are
+ * borrowed and must outlive the handle. */
+ic_cache_t* ic_cache_create_ex(int32_t dim, int64_t capacity, const ic_cache_opts_t* opts);
+
+/*
+ * Append n embeddings and their ids at slots [size, size+n) (paper: update_cache after the
+ * response is served).  emb: [n, dim] in the handle's input dtype; fp32 is rounded to bf16,
+ * round-to-nearest-even, after the optional fp32 L2 normalisation (a zero row stays zero).
+ * ids: [n] int64, opaque to the library, not checked for uniqueness.
+ * n == 0 is a no-op.  IC_ERR_FULL if size + n > capacity, IC_ERR_INVALID for n < 0 or a NULL
+ * or host pointer with n > 0.
+ */
+int ic_cache_insert(ic_cache_t* c, const void* emb, const int64_t* ids, int64_t n);
+
+/*
+ * For each of nq query embeddings return the k entries with the largest score.
+ * q: [nq, dim] in the handle's input dtype (rounded to bf16 like inserted rows).
+ * out_ids [nq, k] int64, out_scores [nq, k] fp32: each row sorted by score descending, equal
+ * scores ordered by earlier insertion; when k exceeds the number of entries the tail is
+ * id -1, score -infinity.  1 <= k <= IC_MAX_K; nq == 0 is a no-op.
+ * Every score comes from an exhaustive pass over all entries: the result is the exact top-k
+ * of the fp32-accumulated scores (no clustering or other approximation).
+ * May grow the library's scratch buffers on the first call with a larger nq or k (this
+ * synchronises the stream); later calls of the same or smaller shape allocate nothing.
+ */
+int ic_cache_query(ic_cache_t* c, const void* q, int32_t nq, int32_t k, int64_t* out_ids,
+                   float* out_scores);
+
+/*
+ * ic_cache_query for callers whose buffers live in HOST memory (pinned memory makes the
+ * copies asynchronous): copies q to the device, runs the query, copies both results back
+ * and synchronises the stream before returning.
+ */
+int ic_cache_query_host(ic_cache_t* c, const void* q_host, int32_t nq, int32_t k,
+                        int64_t* out_ids_host, float* out_scores_host);
+
+/* ic_cache_insert for HOST buffers; synchronises the stream before returning. */
+int ic_cache_insert_host(ic_cache_t* c, const void* emb_host, const int64_t* ids_host, int64_t n);
+
+/* Release the handle and everything the library allocated for it.  NULL is a no-op. */
+void ic_cache_destroy(ic_cache_t* c);
+
+/* Bind the handle to another stream (a cudaStream_t; NULL = legacy default stream).  Work
+ * already enqueued stays on the old stream; ordering between the two is the caller's. */
+int ic_cache_set_stream(ic_cache_t* c, void* cuda_stream);
+
+/* Force a kernel path for later queries (IC_PATH_AUTO restores the default choice).  A
+ * query whose shape the forced path cannot serve returns IC_ERR_UNSUPPORTED. */
+int ic_cache_set_path(ic_cache_t* c, int32_t path);
+
+/* Number of entries inserted so far, or a negative ic_status for a NULL handle. */
+int64_t ic_cache_size(const ic_cache_t* c);
+
+/* Forget all entries (size becomes 0); the slab is not cleared.  Stream-ordered. */
+int ic_cache_clear(ic_cache_t* c);
+
+/* Synchronise the handle's stream and report IC_ERR_TIMEOUT if any kernel since the last
+ * call of this function gave up on a bounded wait, IC_ERR_CUDA on a CUDA error, else IC_OK. */
+int ic_cache_sync(ic_cache_t* c);
+
+/* Kernels launched by this handle so far (insert, query preparation, scoring, merge). */
+int64_t ic_cache_launch_count(const ic_cache_t* c);
+
+/*
+ * The launch plan the library would use for a query of nq vectors, k results, over n entries
+ * of dimension dim on a device with sm_count multiprocessors and smem_optin bytes of opt-in
+ * shared memory per block.  path = IC_PATH_AUTO or a forced ic_path.  Touches no device.
+ * Returns IC_OK, IC_ERR_INVALID or IC_ERR_UNSUPPORTED.
+ */
+int ic_cache_plan(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32_t sm_count,
+                  int32_t smem_optin, ic_cache_plan_t* plan);
+
+/* Message for the most recent failure on the calling thread ("" if none). */
+const char* ic_cache_last_error(void);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int32_t ic_cache_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IC_CACHE_H_ */

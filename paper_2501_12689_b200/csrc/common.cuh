@@ -1,0 +1,120 @@
+// Device helpers shared by the scoring and merge kernels: the packed (score, slot) key and
+// the warp-cooperative sorted insert that every partial top-k list uses.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace icc {
+
+constexpr unsigned FULL_MASK = 0xffffffffu;
+constexpr uint64_t KEY_EMPTY = 0ull;  // smaller than every real key
+
+// Status word values written by kernels whose bounded waits expire (device -> host).
+enum : int { DEV_OK = 0, DEV_TIMEOUT_LOCK = 1, DEV_TIMEOUT_MBAR = 2 };
+
+// Monotone map from fp32 scores to unsigned integers (-0 is folded onto +0 first so that
+// equal scores give equal keys).
+__device__ __forceinline__ uint32_t score_to_ord(float s) {
+  s += 0.0f;
+  uint32_t u = __float_as_uint(s);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float ord_to_score(uint32_t o) {
+  uint32_t u = (o & 0x80000000u) ? (o & 0x7fffffffu) : ~o;
+  return __uint_as_float(u);
+}
+// One 64-bit key per candidate: larger key = better candidate (higher score; on equal score
+// the earlier slot).  A single integer compare therefore orders candidates everywhere.
+__device__ __forceinline__ uint64_t make_key(float score, uint32_t slot) {
+  return ((uint64_t)score_to_ord(score) << 32) | (uint64_t)(0xffffffffu - slot);
+}
+__device__ __forceinline__ uint32_t key_slot(uint64_t key) { return 0xffffffffu - (uint32_t)key; }
+__device__ __forceinline__ float key_score(uint64_t key) { return ord_to_score((uint32_t)(key >> 32)); }
+
+constexpr int MAX_K = 128;  // must equal IC_MAX_K
+
+// Record that a bounded wait expired.  The status word lives in mapped pinned host memory,
+// so a plain store followed by a system-scope fence is what the host polls.
+__device__ __forceinline__ void report_status(int* dev_status, int code) {
+  *reinterpret_cast<volatile int*>(dev_status) = code;
+  __threadfence_system();
+}
+
+// Insert `key` into a descending list of k entries in shared memory, dropping the last one.
+// All 32 lanes of the warp call this with the same arguments; the caller guarantees that no
+// other warp touches the list meanwhile.  A key not larger than the last entry changes
+// nothing.  Returns the new last entry (the list's admission threshold).
+__device__ __forceinline__ uint64_t warp_sorted_insert(uint64_t* list, int k, uint64_t key, int lane) {
+  uint64_t nv[MAX_K / 32];
+#pragma unroll
+  for (int t = 0; t < MAX_K / 32; ++t) {
+    const int i = t * 32 + lane;
+    nv[t] = 0;
+    if (i < k) {
+      const uint64_t cur = list[i];
+      const uint64_t prev = (i > 0) ? list[i - 1] : ~0ull;
+      nv[t] = (cur > key) ? cur : ((prev > key) ? key : prev);
+    }
+  }
+  __syncwarp();
+#pragma unroll
+  for (int t = 0; t < MAX_K / 32; ++t) {
+    const int i = t * 32 + lane;
+    if (i < k) list[i] = nv[t];
+  }
+  __syncwarp();
+  return list[k - 1];
+}
+
+constexpr int LOCK_SPIN_LIMIT = 1 << 22;
+
+// warp_sorted_insert under a per-list spin lock, for lists shared by the warps of a CTA.
+// The wait is bounded: if the lock cannot be taken the candidate is dropped and the status
+// word records it.  All 32 lanes call this with the same arguments.
+__device__ __forceinline__ void locked_insert(uint64_t* list, int k, int* lock, uint64_t key,
+                                              int lane, int* dev_status) {
+  int ok = 1;
+  if (lane == 0) {
+    int spins = 0;
+    while (atomicCAS(lock, 0, 1) != 0) {
+      if (++spins > LOCK_SPIN_LIMIT) {
+        ok = 0;
+        break;
+      }
+      __nanosleep(32);
+    }
+  }
+  ok = __shfl_sync(FULL_MASK, ok, 0);
+  if (!ok) {
+    if (lane == 0) report_status(dev_status, DEV_TIMEOUT_LOCK);
+    return;
+  }
+  __threadfence_block();
+  warp_sorted_insert(list, k, key, lane);
+  __threadfence_block();
+  if (lane == 0) atomicExch(lock, 0);
+}
+
+// Unpack eight bf16 values held in a 16-byte vector into fp32.
+__device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float* x) {
+  x[0] = __uint_as_float(v.x << 16);
+  x[1] = __uint_as_float(v.x & 0xffff0000u);
+  x[2] = __uint_as_float(v.y << 16);
+  x[3] = __uint_as_float(v.y & 0xffff0000u);
+  x[4] = __uint_as_float(v.z << 16);
+  x[5] = __uint_as_float(v.z & 0xffff0000u);
+  x[6] = __uint_as_float(v.w << 16);
+  x[7] = __uint_as_float(v.w & 0xffff0000u);
+}
+
+// Streaming 16-byte global load that does not allocate in L1.
+__device__ __forceinline__ uint4 ld_stream_16B(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+}  // namespace icc

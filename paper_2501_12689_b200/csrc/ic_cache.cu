@@ -1,0 +1,604 @@
+// Host side of the C ABI declared in include/ic_cache.h: argument checking, buffer ownership,
+// launch planning and kernel sequencing.  All arithmetic of the retrieval path runs in the
+// kernels; nothing here touches embedding data on the CPU.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+
+#include "../../include/ic_cache.h"
+#include "kernels.h"
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+int fail(int code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof g_err, fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+constexpr int WINDOW_MAX_NQ = 1024;   // queries scored per pass over the slab
+constexpr int QUERY_TILE = 128;       // tcgen05 path: queries per CTA (MMA M)
+constexpr int ROW_TILE = 256;         // tcgen05 path: cache rows per accumulator (MMA N)
+constexpr int K_CHUNK = 64;           // tcgen05 path: bf16 elements per 128-byte swizzled row
+constexpr int UMMA_STAGE_BYTES = (QUERY_TILE + ROW_TILE) * K_CHUNK * 2;  // 48 KiB
+constexpr int SCAN_MAX_Q = 4;
+constexpr int SCAN_MAX_DIM = 1024;
+constexpr int SCAN_ROWS_PER_STAGE = 32;
+constexpr int GENERIC_QB = 4;
+
+struct DeviceGuard {
+  int prev = -1;
+  bool changed = false;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) changed = (cudaSetDevice(dev) == cudaSuccess);
+  }
+  ~DeviceGuard() {
+    if (changed) cudaSetDevice(prev);
+  }
+};
+
+struct Buffer {
+  void* p = nullptr;
+  size_t bytes = 0;
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+}  // namespace
+
+struct ic_cache {
+  int device = 0;
+  int dim = 0;
+  int64_t capacity = 0;
+  int64_t size = 0;
+  int input_dtype = IC_BF16;
+  int normalize = 0;
+  int forced_path = IC_PATH_AUTO;
+  int sm_count = 0;
+  int smem_optin = 0;
+  cudaStream_t stream = nullptr;
+  void* slab = nullptr;
+  bool own_slab = false;
+  int64_t* ids = nullptr;
+  bool own_ids = false;
+  Buffer q_bf16, q_f32, partials, stage_in, stage_ids, stage_scores;
+  int* h_status = nullptr;  // pinned, mapped; kernels write a code when a bounded wait expires
+  int* d_status = nullptr;
+  int64_t launches = 0;
+  EncodeTiledFn encode = nullptr;
+  CUtensorMap tmap_slab;
+  bool have_tmap_slab = false;
+};
+
+namespace {
+
+size_t in_elem_bytes(const ic_cache* c) { return c->input_dtype == IC_F32 ? 4 : 2; }
+
+bool is_device_ptr(const void* p, int device) {
+  cudaPointerAttributes a;
+  if (cudaPointerGetAttributes(&a, p) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  if (a.type == cudaMemoryTypeManaged) return true;
+  return a.type == cudaMemoryTypeDevice && a.device == device;
+}
+
+int ensure(ic_cache* c, Buffer& b, size_t bytes, const char* what) {
+  if (bytes <= b.bytes) return IC_OK;
+  if (b.p) {
+    // the old buffer may still be in use by enqueued work
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(IC_ERR_CUDA, "stream sync failed while growing %s", what);
+    cudaFree(b.p);
+    b.p = nullptr;
+    b.bytes = 0;
+  }
+  cudaError_t e = cudaMalloc(&b.p, bytes);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    b.p = nullptr;
+    return fail(IC_ERR_NOMEM, "cudaMalloc of %zu bytes for %s failed: %s", bytes, what, cudaGetErrorString(e));
+  }
+  b.bytes = bytes;
+  return IC_OK;
+}
+
+void release(Buffer& b) {
+  if (b.p) cudaFree(b.p);
+  b.p = nullptr;
+  b.bytes = 0;
+}
+
+int encode_2d(ic_cache* c, CUtensorMap* tm, const void* base, uint64_t rows, uint32_t box_rows) {
+  // [rows, dim] bf16 row-major; box = K_CHUNK elements (128 bytes) x box_rows rows, 128-byte
+  // swizzle; out-of-range elements (row tail, dim tail) read as zero.
+  cuuint64_t dims[2] = {(cuuint64_t)c->dim, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)c->dim * 2};
+  cuuint32_t box[2] = {(cuuint32_t)K_CHUNK, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = c->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                         estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(IC_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+  return IC_OK;
+}
+
+int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32_t sm_count,
+              int32_t smem_optin, ic_cache_plan_t* out) {
+  if (!out) return fail(IC_ERR_INVALID, "plan: NULL output");
+  memset(out, 0, sizeof *out);
+  if (dim < 8 || dim > IC_MAX_DIM || (dim % 8) != 0) return fail(IC_ERR_INVALID, "dim %d must be a multiple of 8 in [8, %d]", dim, IC_MAX_DIM);
+  if (n < 0 || nq < 1 || k < 1 || k > IC_MAX_K) return fail(IC_ERR_INVALID, "plan: need n >= 0, nq >= 1, 1 <= k <= %d", IC_MAX_K);
+  if (sm_count < 1 || smem_optin < 48 * 1024) return fail(IC_ERR_INVALID, "plan: bad device limits");
+  if (path < IC_PATH_AUTO || path > IC_PATH_UMMA) return fail(IC_ERR_INVALID, "plan: unknown path %d", path);
+  const int window = std::min<int>(nq, WINDOW_MAX_NQ);
+  const int n_windows = (nq + WINDOW_MAX_NQ - 1) / WINDOW_MAX_NQ;
+  if (path == IC_PATH_AUTO) path = (nq <= SCAN_MAX_Q && dim <= SCAN_MAX_DIM) ? IC_PATH_SCAN : IC_PATH_UMMA;
+  out->path = path;
+  const int merge_lists_max = (smem_optin - 4096) / (k * 8 + 4);
+  if (path == IC_PATH_GENERIC) {
+    out->query_tile = GENERIC_QB;
+    out->n_query_tiles = (window + GENERIC_QB - 1) / GENERIC_QB;
+    out->n_partitions = std::max(1, std::min(2 * sm_count, merge_lists_max));
+    out->n_ctas = out->n_partitions;
+    out->n_stages = 0;
+    out->smem_bytes = GENERIC_QB * k * 8 + 64;
+    out->n_launches = n_windows * out->n_query_tiles;
+  } else if (path == IC_PATH_SCAN) {
+    if (dim > SCAN_MAX_DIM) return fail(IC_ERR_UNSUPPORTED, "scan path needs dim <= %d", SCAN_MAX_DIM);
+    out->query_tile = window <= 1 ? 1 : (window <= 2 ? 2 : SCAN_MAX_Q);
+    out->n_query_tiles = (window + out->query_tile - 1) / out->query_tile;
+    out->n_partitions = std::max(1, std::min(sm_count, merge_lists_max));
+    out->n_ctas = out->n_partitions;
+    const int stage_bytes = SCAN_ROWS_PER_STAGE * dim * 2;
+    const int fixed = 2048 + SCAN_MAX_Q * k * 8;
+    out->n_stages = std::min(8, (smem_optin - fixed) / stage_bytes);
+    if (out->n_stages < 2) return fail(IC_ERR_UNSUPPORTED, "scan path: shared memory too small for dim %d", dim);
+    out->smem_bytes = fixed + out->n_stages * stage_bytes;
+    out->n_launches = n_windows * out->n_query_tiles;
+  } else {
+    out->query_tile = QUERY_TILE;
+    out->n_query_tiles = (window + QUERY_TILE - 1) / QUERY_TILE;
+    out->n_partitions = std::max(1, std::min(sm_count / out->n_query_tiles, merge_lists_max));
+    out->n_ctas = out->n_partitions * out->n_query_tiles;
+    const int fixed = 2048 + QUERY_TILE * k * 8;   // 1 KiB alignment slack + barriers, lists
+    out->n_stages = std::min(6, (smem_optin - fixed) / UMMA_STAGE_BYTES);
+    if (out->n_stages < 2) return fail(IC_ERR_UNSUPPORTED, "tensor-core path: shared memory too small");
+    out->smem_bytes = fixed + out->n_stages * UMMA_STAGE_BYTES;
+    out->n_launches = n_windows;
+  }
+  return IC_OK;
+}
+
+int check_timeout(ic_cache* c) {
+  if (c->h_status && *reinterpret_cast<volatile int*>(c->h_status) != 0)
+    return fail(IC_ERR_TIMEOUT, "an earlier kernel gave up on a bounded wait (code %d); call ic_cache_sync to clear", *c->h_status);
+  return IC_OK;
+}
+
+int do_insert(ic_cache* c, const void* emb, const int64_t* ids, int64_t n) {
+  cudaError_t e = icc::launch_convert_rows(emb, c->input_dtype == IC_F32, n, c->dim, c->normalize,
+                                           static_cast<char*>(c->slab) + (size_t)c->size * c->dim * 2, nullptr, n,
+                                           c->stream);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "insert kernel launch failed: %s", cudaGetErrorString(e));
+  c->launches += 1;
+  e = cudaMemcpyAsync(c->ids + c->size, ids, (size_t)n * 8, cudaMemcpyDeviceToDevice, c->stream);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "id copy failed: %s", cudaGetErrorString(e));
+  c->size += n;
+  return IC_OK;
+}
+
+// One window of at most WINDOW_MAX_NQ queries, all pointers on the device.
+int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids, float* out_scores) {
+  ic_cache_plan_t pl;
+  int rc = plan_impl(c->dim, c->size, nq, k, c->forced_path, c->sm_count, c->smem_optin, &pl);
+  if (rc != IC_OK) return rc;
+  const int nq_pad = (nq + QUERY_TILE - 1) / QUERY_TILE * QUERY_TILE;
+  if ((rc = ensure(c, c->q_bf16, (size_t)nq_pad * c->dim * 2, "query staging (bf16)")) != IC_OK) return rc;
+  if ((rc = ensure(c, c->q_f32, (size_t)nq * c->dim * 4, "query staging (fp32)")) != IC_OK) return rc;
+  if ((rc = ensure(c, c->partials, (size_t)pl.n_partitions * nq * k * 8, "partial top-k lists")) != IC_OK) return rc;
+
+  cudaError_t e = icc::launch_convert_rows(q, c->input_dtype == IC_F32, nq, c->dim, c->normalize, c->q_bf16.p,
+                                           static_cast<float*>(c->q_f32.p), nq_pad, c->stream);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "query preparation launch failed: %s", cudaGetErrorString(e));
+  c->launches += 1;
+  uint64_t* partials = static_cast<uint64_t*>(c->partials.p);
+
+  if (pl.path == IC_PATH_GENERIC) {
+    for (int q0 = 0; q0 < nq; q0 += GENERIC_QB) {
+      e = icc::launch_generic(c->slab, c->size, c->dim, static_cast<const float*>(c->q_f32.p), q0, nq, k,
+                              partials, pl.n_partitions, pl.smem_bytes, c->d_status, c->stream);
+      if (e != cudaSuccess) return fail(IC_ERR_CUDA, "generic scoring launch failed: %s", cudaGetErrorString(e));
+      c->launches += 1;
+    }
+  } else if (pl.path == IC_PATH_SCAN) {
+    for (int q0 = 0; q0 < nq; q0 += pl.query_tile) {
+      icc::ScanParams sp;
+      sp.slab = c->slab;
+      sp.n = c->size;
+      sp.dim = c->dim;
+      sp.q_f32 = static_cast<const float*>(c->q_f32.p);
+      sp.q0 = q0;
+      sp.nq = nq;
+      sp.qb = pl.query_tile;
+      sp.k = k;
+      sp.partials = partials;
+      sp.n_part = pl.n_partitions;
+      sp.n_stages = pl.n_stages;
+      sp.rows_per_stage = SCAN_ROWS_PER_STAGE;
+      sp.smem_bytes = pl.smem_bytes;
+      sp.dev_status = c->d_status;
+      e = icc::launch_scan(sp, c->stream);
+      if (e != cudaSuccess) return fail(IC_ERR_CUDA, "scan launch failed: %s", cudaGetErrorString(e));
+      c->launches += 1;
+    }
+  } else {
+    if (!c->have_tmap_slab) return fail(IC_ERR_UNSUPPORTED, "tensor-core path unavailable: no tensor map for the slab");
+    icc::UmmaParams up;
+    if ((rc = encode_2d(c, &up.tmap_q, c->q_bf16.p, (uint64_t)nq_pad, QUERY_TILE)) != IC_OK) return rc;
+    up.tmap_slab = c->tmap_slab;
+    up.n = c->size;
+    up.dim = c->dim;
+    up.q0 = 0;
+    up.nq = nq;
+    up.k = k;
+    up.n_query_tiles = pl.n_query_tiles;
+    up.n_part = pl.n_partitions;
+    up.n_stages = pl.n_stages;
+    up.smem_bytes = pl.smem_bytes;
+    up.partials = partials;
+    up.dev_status = c->d_status;
+    e = icc::launch_umma(up, c->stream);
+    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core scoring launch failed: %s", cudaGetErrorString(e));
+    c->launches += 1;
+  }
+  e = icc::launch_merge(partials, pl.n_partitions, nq, k, c->ids, out_ids, out_scores, c->stream);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "merge launch failed: %s", cudaGetErrorString(e));
+  c->launches += 1;
+  return IC_OK;
+}
+
+int check_query_args(ic_cache* c, const void* q, int32_t nq, int32_t k, const void* out_ids, const void* out_scores) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  if (nq < 0) return fail(IC_ERR_INVALID, "nq %d < 0", nq);
+  if (k < 1 || k > IC_MAX_K) return fail(IC_ERR_INVALID, "k %d outside [1, %d]", k, IC_MAX_K);
+  if (nq > 0 && (!q || !out_ids || !out_scores)) return fail(IC_ERR_INVALID, "NULL pointer with nq > 0");
+  return IC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* ic_cache_last_error(void) { return g_err; }
+
+int32_t ic_cache_version(void) { return 100; }
+
+int ic_cache_plan(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32_t sm_count,
+                  int32_t smem_optin, ic_cache_plan_t* plan) {
+  return plan_impl(dim, n, nq, k, path, sm_count, smem_optin, plan);
+}
+
+ic_cache_t* ic_cache_create(int32_t dim, int64_t capacity) { return ic_cache_create_ex(dim, capacity, nullptr); }
+
+ic_cache_t* ic_cache_create_ex(int32_t dim, int64_t capacity, const ic_cache_opts_t* opts) {
+  g_err[0] = 0;
+  if (dim < 8 || dim > IC_MAX_DIM || (dim % 8) != 0) {
+    fail(IC_ERR_INVALID, "dim %d must be a multiple of 8 in [8, %d]", dim, IC_MAX_DIM);
+    return nullptr;
+  }
+  if (capacity < 1 || capacity > 0xfffffffell) {
+    fail(IC_ERR_INVALID, "capacity %lld outside [1, 2^32-2]", (long long)capacity);
+    return nullptr;
+  }
+  ic_cache_opts_t o;
+  memset(&o, 0, sizeof o);
+  o.device = -1;
+  if (opts) {
+    if (opts->struct_size < sizeof(uint32_t) || opts->struct_size > sizeof o) {
+      fail(IC_ERR_INVALID, "opts.struct_size %u not understood (this build: %zu)", opts->struct_size, sizeof o);
+      return nullptr;
+    }
+    memcpy(&o, opts, opts->struct_size);
+  }
+  if (o.input_dtype != IC_BF16 && o.input_dtype != IC_F32) {
+    fail(IC_ERR_INVALID, "unknown input_dtype %d", o.input_dtype);
+    return nullptr;
+  }
+  int ndev = 0;
+  cudaError_t e = cudaGetDeviceCount(&ndev);
+  if (e != cudaSuccess || ndev == 0) {
+    cudaGetLastError();
+    fail(IC_ERR_CUDA, "no usable CUDA device (%s); this library has no CPU fallback",
+         e != cudaSuccess ? cudaGetErrorString(e) : "device count is 0");
+    return nullptr;
+  }
+  int dev = o.device;
+  if (dev < 0 && cudaGetDevice(&dev) != cudaSuccess) {
+    fail(IC_ERR_CUDA, "cudaGetDevice failed");
+    return nullptr;
+  }
+  if (dev >= ndev) {
+    fail(IC_ERR_INVALID, "device %d does not exist (%d devices)", dev, ndev);
+    return nullptr;
+  }
+  DeviceGuard guard(dev);
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+    fail(IC_ERR_CUDA, "cudaGetDeviceProperties failed");
+    return nullptr;
+  }
+  if (prop.major != 10) {
+    fail(IC_ERR_UNSUPPORTED, "device %d is sm_%d%d; this library is built for sm_100a only", dev, prop.major, prop.minor);
+    return nullptr;
+  }
+  ic_cache* c = new (std::nothrow) ic_cache();
+  if (!c) {
+    fail(IC_ERR_NOMEM, "host allocation failed");
+    return nullptr;
+  }
+  c->device = dev;
+  c->dim = dim;
+  c->capacity = capacity;
+  c->input_dtype = o.input_dtype;
+  c->normalize = o.normalize ? 1 : 0;
+  c->stream = static_cast<cudaStream_t>(o.stream);
+  c->sm_count = prop.multiProcessorCount;
+  c->smem_optin = (int)prop.sharedMemPerBlockOptin;
+
+  bool ok = true;
+  if (o.slab) {
+    if (!is_device_ptr(o.slab, dev) || (reinterpret_cast<uintptr_t>(o.slab) & 255)) {
+      fail(IC_ERR_INVALID, "opts.slab must be a 256-byte aligned device pointer on device %d", dev);
+      ok = false;
+    }
+    c->slab = o.slab;
+  } else {
+    e = cudaMalloc(&c->slab, (size_t)capacity * dim * 2);
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      fail(IC_ERR_NOMEM, "cudaMalloc of the %zu-byte slab failed: %s", (size_t)capacity * dim * 2, cudaGetErrorString(e));
+      c->slab = nullptr;
+      ok = false;
+    }
+    c->own_slab = ok;
+  }
+  if (ok) {
+    if (o.ids) {
+      if (!is_device_ptr(o.ids, dev)) {
+        fail(IC_ERR_INVALID, "opts.ids must be a device pointer on device %d", dev);
+        ok = false;
+      }
+      c->ids = static_cast<int64_t*>(o.ids);
+    } else {
+      e = cudaMalloc(reinterpret_cast<void**>(&c->ids), (size_t)capacity * 8);
+      if (e != cudaSuccess) {
+        cudaGetLastError();
+        fail(IC_ERR_NOMEM, "cudaMalloc of the id array failed: %s", cudaGetErrorString(e));
+        c->ids = nullptr;
+        ok = false;
+      }
+      c->own_ids = ok;
+    }
+  }
+  if (ok) {
+    e = cudaHostAlloc(reinterpret_cast<void**>(&c->h_status), sizeof(int), cudaHostAllocMapped);
+    if (e == cudaSuccess) {
+      *c->h_status = 0;
+      e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->d_status), c->h_status, 0);
+    }
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      fail(IC_ERR_CUDA, "status word allocation failed: %s", cudaGetErrorString(e));
+      ok = false;
+    }
+  }
+  if (ok) {
+    cudaDriverEntryPointQueryResult qres;
+    void* fn = nullptr;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+      cudaGetLastError();
+      fail(IC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+      ok = false;
+    } else {
+      c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+      ok = encode_2d(c, &c->tmap_slab, c->slab, (uint64_t)capacity, ROW_TILE) == IC_OK;
+      c->have_tmap_slab = ok;
+    }
+  }
+  if (ok) {
+    cudaError_t e1 = icc::merge_configure(c->smem_optin);
+    cudaError_t e2 = icc::scan_configure(c->smem_optin);
+    cudaError_t e3 = icc::umma_configure(c->smem_optin);
+    if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess) {
+      cudaGetLastError();
+      fail(IC_ERR_CUDA, "kernel attribute set-up failed (merge %d, scan %d, tensor-core %d)", (int)e1, (int)e2, (int)e3);
+      ok = false;
+    }
+  }
+  if (!ok) {
+    char keep[sizeof g_err];
+    memcpy(keep, g_err, sizeof keep);
+    ic_cache_destroy(c);
+    memcpy(g_err, keep, sizeof keep);
+    return nullptr;
+  }
+  return c;
+}
+
+void ic_cache_destroy(ic_cache_t* c) {
+  if (!c) return;
+  DeviceGuard guard(c->device);
+  cudaStreamSynchronize(c->stream);
+  if (c->own_slab && c->slab) cudaFree(c->slab);
+  if (c->own_ids && c->ids) cudaFree(c->ids);
+  release(c->q_bf16);
+  release(c->q_f32);
+  release(c->partials);
+  release(c->stage_in);
+  release(c->stage_ids);
+  release(c->stage_scores);
+  if (c->h_status) cudaFreeHost(c->h_status);
+  cudaGetLastError();
+  delete c;
+}
+
+int ic_cache_insert(ic_cache_t* c, const void* emb, const int64_t* ids, int64_t n) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  if (n < 0) return fail(IC_ERR_INVALID, "n %lld < 0", (long long)n);
+  if (n == 0) return IC_OK;
+  if (!emb || !ids) return fail(IC_ERR_INVALID, "NULL pointer with n > 0");
+  if (c->size + n > c->capacity)
+    return fail(IC_ERR_FULL, "insert of %lld rows exceeds capacity (%lld of %lld used)", (long long)n, (long long)c->size, (long long)c->capacity);
+  DeviceGuard guard(c->device);
+  if (!is_device_ptr(emb, c->device) || !is_device_ptr(ids, c->device))
+    return fail(IC_ERR_INVALID, "emb and ids must be device pointers on device %d (use ic_cache_insert_host for host memory)", c->device);
+  int rc = check_timeout(c);
+  if (rc != IC_OK) return rc;
+  return do_insert(c, emb, ids, n);
+}
+
+int ic_cache_insert_host(ic_cache_t* c, const void* emb_host, const int64_t* ids_host, int64_t n) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  if (n < 0) return fail(IC_ERR_INVALID, "n %lld < 0", (long long)n);
+  if (n == 0) return IC_OK;
+  if (!emb_host || !ids_host) return fail(IC_ERR_INVALID, "NULL pointer with n > 0");
+  if (c->size + n > c->capacity)
+    return fail(IC_ERR_FULL, "insert of %lld rows exceeds capacity (%lld of %lld used)", (long long)n, (long long)c->size, (long long)c->capacity);
+  DeviceGuard guard(c->device);
+  int rc = check_timeout(c);
+  if (rc != IC_OK) return rc;
+  // stage in slices so that a large bulk load needs only a bounded device buffer
+  const int64_t slice = std::max<int64_t>(1, (int64_t)(64u << 20) / ((int64_t)c->dim * (int64_t)in_elem_bytes(c)));
+  const size_t row_bytes = (size_t)c->dim * in_elem_bytes(c);
+  if ((rc = ensure(c, c->stage_in, (size_t)std::min(slice, n) * row_bytes, "insert staging")) != IC_OK) return rc;
+  if ((rc = ensure(c, c->stage_ids, (size_t)std::min(slice, n) * 8, "insert id staging")) != IC_OK) return rc;
+  const int64_t size_before = c->size;
+  for (int64_t r0 = 0; r0 < n; r0 += slice) {
+    const int64_t rows = std::min(slice, n - r0);
+    cudaError_t e = cudaMemcpyAsync(c->stage_in.p, static_cast<const char*>(emb_host) + (size_t)r0 * row_bytes,
+                                    (size_t)rows * row_bytes, cudaMemcpyHostToDevice, c->stream);
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(c->stage_ids.p, ids_host + r0, (size_t)rows * 8, cudaMemcpyHostToDevice, c->stream);
+    if (e != cudaSuccess) {
+      c->size = size_before;
+      return fail(IC_ERR_CUDA, "host-to-device copy failed: %s", cudaGetErrorString(e));
+    }
+    rc = do_insert(c, c->stage_in.p, static_cast<const int64_t*>(c->stage_ids.p), rows);
+    if (rc != IC_OK) {
+      c->size = size_before;
+      return rc;
+    }
+    if (r0 + slice < n && cudaStreamSynchronize(c->stream) != cudaSuccess) {  // staging is reused
+      c->size = size_before;
+      return fail(IC_ERR_CUDA, "stream sync failed during host insert");
+    }
+  }
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) {
+    c->size = size_before;
+    return fail(IC_ERR_CUDA, "stream sync failed after host insert");
+  }
+  return IC_OK;
+}
+
+int ic_cache_query(ic_cache_t* c, const void* q, int32_t nq, int32_t k, int64_t* out_ids, float* out_scores) {
+  int rc = check_query_args(c, q, nq, k, out_ids, out_scores);
+  if (rc != IC_OK || nq == 0) return rc;
+  DeviceGuard guard(c->device);
+  if (!is_device_ptr(q, c->device) || !is_device_ptr(out_ids, c->device) || !is_device_ptr(out_scores, c->device))
+    return fail(IC_ERR_INVALID, "q, out_ids and out_scores must be device pointers on device %d (use ic_cache_query_host for host memory)", c->device);
+  if ((rc = check_timeout(c)) != IC_OK) return rc;
+  const size_t q_row = (size_t)c->dim * in_elem_bytes(c);
+  for (int q0 = 0; q0 < nq; q0 += WINDOW_MAX_NQ) {
+    const int w = std::min(WINDOW_MAX_NQ, nq - q0);
+    rc = do_query_window(c, static_cast<const char*>(q) + (size_t)q0 * q_row, w, k, out_ids + (size_t)q0 * k,
+                         out_scores + (size_t)q0 * k);
+    if (rc != IC_OK) return rc;
+  }
+  return IC_OK;
+}
+
+int ic_cache_query_host(ic_cache_t* c, const void* q_host, int32_t nq, int32_t k, int64_t* out_ids_host,
+                        float* out_scores_host) {
+  int rc = check_query_args(c, q_host, nq, k, out_ids_host, out_scores_host);
+  if (rc != IC_OK || nq == 0) return rc;
+  DeviceGuard guard(c->device);
+  if ((rc = check_timeout(c)) != IC_OK) return rc;
+  const size_t q_bytes = (size_t)nq * c->dim * in_elem_bytes(c);
+  if ((rc = ensure(c, c->stage_in, q_bytes, "query input staging")) != IC_OK) return rc;
+  if ((rc = ensure(c, c->stage_ids, (size_t)nq * k * 8, "result id staging")) != IC_OK) return rc;
+  if ((rc = ensure(c, c->stage_scores, (size_t)nq * k * 4, "result score staging")) != IC_OK) return rc;
+  cudaError_t e = cudaMemcpyAsync(c->stage_in.p, q_host, q_bytes, cudaMemcpyHostToDevice, c->stream);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "host-to-device copy failed: %s", cudaGetErrorString(e));
+  const size_t q_row = (size_t)c->dim * in_elem_bytes(c);
+  for (int q0 = 0; q0 < nq; q0 += WINDOW_MAX_NQ) {
+    const int w = std::min(WINDOW_MAX_NQ, nq - q0);
+    rc = do_query_window(c, static_cast<const char*>(c->stage_in.p) + (size_t)q0 * q_row, w, k,
+                         static_cast<int64_t*>(c->stage_ids.p) + (size_t)q0 * k,
+                         static_cast<float*>(c->stage_scores.p) + (size_t)q0 * k);
+    if (rc != IC_OK) return rc;
+  }
+  e = cudaMemcpyAsync(out_ids_host, c->stage_ids.p, (size_t)nq * k * 8, cudaMemcpyDeviceToHost, c->stream);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(out_scores_host, c->stage_scores.p, (size_t)nq * k * 4, cudaMemcpyDeviceToHost, c->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "result copy failed: %s", cudaGetErrorString(e));
+  return check_timeout(c);
+}
+
+int ic_cache_set_stream(ic_cache_t* c, void* cuda_stream) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  c->stream = static_cast<cudaStream_t>(cuda_stream);
+  return IC_OK;
+}
+
+int ic_cache_set_path(ic_cache_t* c, int32_t path) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  if (path < IC_PATH_AUTO || path > IC_PATH_UMMA) return fail(IC_ERR_INVALID, "unknown path %d", path);
+  c->forced_path = path;
+  return IC_OK;
+}
+
+int64_t ic_cache_size(const ic_cache_t* c) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  return c->size;
+}
+
+int ic_cache_clear(ic_cache_t* c) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  c->size = 0;
+  return IC_OK;
+}
+
+int ic_cache_sync(ic_cache_t* c) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  DeviceGuard guard(c->device);
+  cudaError_t e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "stream sync failed: %s", cudaGetErrorString(e));
+  if (c->h_status && *reinterpret_cast<volatile int*>(c->h_status) != 0) {
+    const int code = *c->h_status;
+    *c->h_status = 0;
+    return fail(IC_ERR_TIMEOUT, "a kernel gave up on a bounded wait (code %d); its results are incomplete", code);
+  }
+  return IC_OK;
+}
+
+int64_t ic_cache_launch_count(const ic_cache_t* c) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  return c->launches;
+}
+
+}  // extern "C"

@@ -1,0 +1,60 @@
+// Host-side launchers of the library's kernels (internal to the shared library).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace icc {
+
+// Convert/normalise `nrows` input rows ([nrows, dim], fp32 if in_is_f32 else bf16) into bf16
+// rows at out_bf16 (row pitch = dim elements).  Rows nrows .. pad_rows-1 of out_bf16 are set
+// to zero.  If out_f32 != NULL it receives the stored bf16 values widened to fp32.
+cudaError_t launch_convert_rows(const void* in, int in_is_f32, int64_t nrows, int dim, int normalize,
+                                void* out_bf16, float* out_f32, int64_t pad_rows, cudaStream_t st);
+
+// Generic CUDA-core scoring of up to 4 queries [q0, q0+4) against rows [0, n).
+// partials: [n_part][nq][k] packed keys.
+cudaError_t launch_generic(const void* slab, int64_t n, int dim, const float* q_f32, int q0, int nq,
+                           int k, uint64_t* partials, int n_part, int smem_bytes, int* dev_status,
+                           cudaStream_t st);
+
+// Bulk-copy staged scan: qb in {1,2,4} queries starting at q0.
+struct ScanParams {
+  const void* slab;
+  int64_t n;
+  int dim;
+  const float* q_f32;
+  int q0, nq, qb, k;
+  uint64_t* partials;
+  int n_part;       // = number of CTAs
+  int n_stages;
+  int rows_per_stage;
+  int smem_bytes;
+  int* dev_status;
+};
+cudaError_t launch_scan(const ScanParams& p, cudaStream_t st);
+cudaError_t scan_configure(int smem_optin);
+
+// tcgen05 scoring: query tiles of 128 x row tiles of 256, top-k fused in the epilogue.
+struct UmmaParams {
+  CUtensorMap tmap_q;     // [nq_pad, dim] bf16, box 64 x 128, 128-byte swizzle
+  CUtensorMap tmap_slab;  // [capacity, dim] bf16, box 64 x 256, 128-byte swizzle
+  int64_t n;
+  int dim;
+  int q0, nq, k;          // queries [q0, q0 + n_query_tiles*128) of the staged batch
+  int n_query_tiles;
+  int n_part;
+  int n_stages;
+  int smem_bytes;
+  uint64_t* partials;     // [n_part][nq][k]
+  int* dev_status;
+};
+cudaError_t launch_umma(const UmmaParams& p, cudaStream_t st);
+cudaError_t umma_configure(int smem_optin);
+
+// Merge n_part partial lists per query into the final sorted top-k and gather ids.
+cudaError_t launch_merge(const uint64_t* partials, int n_part, int nq, int k, const int64_t* ids,
+                         int64_t* out_ids, float* out_scores, cudaStream_t st);
+cudaError_t merge_configure(int smem_optin);
+
+}  // namespace icc

@@ -1,0 +1,90 @@
+// Global merge: per query, the top-k of the n_part sorted partial lists, then the id gather.
+// One CTA per query.  The lists are copied to shared memory; warp 0 then runs a k-round
+// tournament over the list heads: each lane keeps the best head among the lists it owns and
+// two warp max-reductions (score word, then slot word) pick the winner of the round.
+#include <math.h>
+
+#include "common.cuh"
+#include "kernels.h"
+
+namespace icc {
+
+constexpr int MERGE_THREADS = 128;
+
+__global__ void __launch_bounds__(MERGE_THREADS)
+merge_topk_kernel(const uint64_t* __restrict__ partials, int n_part, int nq, int k,
+                  const int64_t* __restrict__ ids, int64_t* __restrict__ out_ids,
+                  float* __restrict__ out_scores) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  uint64_t* cand = reinterpret_cast<uint64_t*>(smem_raw);                 // [n_part][k]
+  uint32_t* pos = reinterpret_cast<uint32_t*>(cand + (size_t)n_part * k);  // [n_part]
+  __shared__ uint32_t win_slot[MAX_K];
+  __shared__ float win_score[MAX_K];
+
+  const int q = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
+  const int total = n_part * k;
+  for (int i = tid; i < total; i += MERGE_THREADS) {
+    const int p = i / k, j = i - p * k;
+    cand[i] = partials[((size_t)p * nq + q) * k + j];
+  }
+  for (int p = tid; p < n_part; p += MERGE_THREADS) pos[p] = 0;
+  __syncthreads();
+
+  if (tid < 32) {
+    uint64_t best = KEY_EMPTY;
+    int best_p = -1;
+    for (int p = lane; p < n_part; p += 32) {
+      const uint64_t key = cand[(size_t)p * k];
+      if (key > best) { best = key; best_p = p; }
+    }
+    int r = 0;
+    for (; r < k; ++r) {
+      const uint32_t hi = (uint32_t)(best >> 32);
+      const uint32_t top_hi = __reduce_max_sync(FULL_MASK, hi);
+      if (top_hi == 0) break;  // every list exhausted (warp-uniform)
+      const uint32_t lo = (hi == top_hi) ? (uint32_t)best : 0u;
+      const uint32_t top_lo = __reduce_max_sync(FULL_MASK, lo);
+      if (hi == top_hi && lo == top_lo) {  // keys are unique, so exactly one lane wins
+        win_slot[r] = 0xffffffffu - top_lo;
+        win_score[r] = ord_to_score(top_hi);
+        pos[best_p] += 1;
+        best = KEY_EMPTY;
+        best_p = -1;
+        for (int p = lane; p < n_part; p += 32) {
+          const uint32_t j = pos[p];
+          const uint64_t key = (j < (uint32_t)k) ? cand[(size_t)p * k + j] : KEY_EMPTY;
+          if (key > best) { best = key; best_p = p; }
+        }
+      }
+    }
+    for (int i = r + lane; i < k; i += 32) {  // fewer than k entries in the cache
+      win_slot[i] = 0xffffffffu;
+      win_score[i] = -INFINITY;
+    }
+  }
+  __syncthreads();
+  for (int i = tid; i < k; i += MERGE_THREADS) {
+    const uint32_t slot = win_slot[i];
+    out_scores[(size_t)q * k + i] = win_score[i];
+    out_ids[(size_t)q * k + i] = (slot == 0xffffffffu) ? (int64_t)-1 : ids[slot];
+  }
+}
+
+static int g_merge_smem_limit = 48 * 1024;
+
+cudaError_t merge_configure(int smem_optin) {
+  cudaError_t e = cudaFuncSetAttribute(merge_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       smem_optin - 2048);
+  if (e == cudaSuccess) g_merge_smem_limit = smem_optin - 2048;
+  return e;
+}
+
+cudaError_t launch_merge(const uint64_t* partials, int n_part, int nq, int k, const int64_t* ids,
+                         int64_t* out_ids, float* out_scores, cudaStream_t st) {
+  const size_t smem = (size_t)n_part * k * 8 + (size_t)n_part * 4;
+  if (smem > (size_t)g_merge_smem_limit) return cudaErrorInvalidValue;
+  merge_topk_kernel<<<nq, MERGE_THREADS, smem, st>>>(partials, n_part, nq, k, ids, out_ids, out_scores);
+  return cudaGetLastError();
+}
+
+}  // namespace icc

@@ -1,0 +1,89 @@
+// Row conversion used by insert (into the slab) and by query preparation (into the query
+// staging buffers): optional fp32 L2 normalisation, then round-to-nearest-even to bf16.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace icc {
+
+constexpr int CONV_WARPS = 8;
+constexpr int CONV_MAX_CHUNKS = 16;  // 16 chunks * 32 lanes * 8 elements = 4096 = IC_MAX_DIM
+
+// One warp per row.  Lane l owns the 8-element chunks l, l+32, ... of the row.
+template <bool IN_F32>
+__global__ void __launch_bounds__(CONV_WARPS * 32)
+convert_rows_kernel(const void* __restrict__ in, int64_t nrows, int dim, int normalize,
+                    __nv_bfloat16* __restrict__ out_bf16, float* __restrict__ out_f32,
+                    int64_t pad_rows) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * CONV_WARPS + (threadIdx.x >> 5);
+  if (row >= pad_rows) return;
+  const int nchunk = dim >> 3;
+  uint4* orow = reinterpret_cast<uint4*>(out_bf16 + row * dim);
+  if (row >= nrows) {  // zero padding rows
+    for (int c = lane; c < nchunk; c += 32) orow[c] = make_uint4(0, 0, 0, 0);
+    return;
+  }
+  float x[CONV_MAX_CHUNKS / 1][8];
+  float ss = 0.0f;
+#pragma unroll
+  for (int t = 0; t < CONV_MAX_CHUNKS; ++t) {
+    const int c = t * 32 + lane;
+    if (c < nchunk) {
+      if (IN_F32) {
+        const float4* p = reinterpret_cast<const float4*>(static_cast<const float*>(in) + row * dim) + 2 * c;
+        const float4 a = p[0], b = p[1];
+        x[t][0] = a.x; x[t][1] = a.y; x[t][2] = a.z; x[t][3] = a.w;
+        x[t][4] = b.x; x[t][5] = b.y; x[t][6] = b.z; x[t][7] = b.w;
+      } else {
+        const uint4 v = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(in) + row * dim)[c];
+        bf16x8_to_f32(v, x[t]);
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) ss = fmaf(x[t][e], x[t][e], ss);
+    }
+  }
+  float scale = 1.0f;
+  if (normalize) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(FULL_MASK, ss, o);
+    scale = (ss > 0.0f) ? (1.0f / sqrtf(ss)) : 0.0f;
+  }
+#pragma unroll
+  for (int t = 0; t < CONV_MAX_CHUNKS; ++t) {
+    const int c = t * 32 + lane;
+    if (c < nchunk) {
+      uint32_t w[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat16 lo = __float2bfloat16_rn(x[t][2 * e] * scale);
+        const __nv_bfloat16 hi = __float2bfloat16_rn(x[t][2 * e + 1] * scale);
+        w[e] = (uint32_t)__bfloat16_as_ushort(lo) | ((uint32_t)__bfloat16_as_ushort(hi) << 16);
+      }
+      const uint4 v = make_uint4(w[0], w[1], w[2], w[3]);
+      orow[c] = v;
+      if (out_f32) {
+        float y[8];
+        bf16x8_to_f32(v, y);
+        float4* q = reinterpret_cast<float4*>(out_f32 + row * dim) + 2 * c;
+        q[0] = make_float4(y[0], y[1], y[2], y[3]);
+        q[1] = make_float4(y[4], y[5], y[6], y[7]);
+      }
+    }
+  }
+}
+
+cudaError_t launch_convert_rows(const void* in, int in_is_f32, int64_t nrows, int dim, int normalize,
+                                void* out_bf16, float* out_f32, int64_t pad_rows, cudaStream_t st) {
+  if (pad_rows < nrows) pad_rows = nrows;
+  if (pad_rows == 0) return cudaSuccess;
+  const unsigned blocks = (unsigned)((pad_rows + CONV_WARPS - 1) / CONV_WARPS);
+  if (in_is_f32)
+    convert_rows_kernel<true><<<blocks, CONV_WARPS * 32, 0, st>>>(
+        in, nrows, dim, normalize, static_cast<__nv_bfloat16*>(out_bf16), out_f32, pad_rows);
+  else
+    convert_rows_kernel<false><<<blocks, CONV_WARPS * 32, 0, st>>>(
+        in, nrows, dim, normalize, static_cast<__nv_bfloat16*>(out_bf16), out_f32, pad_rows);
+  return cudaGetLastError();
+}
+
+}  // namespace icc

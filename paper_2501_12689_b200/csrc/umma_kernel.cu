@@ -1,0 +1,241 @@
+// Tensor-core path: scores = Q x X^T on tcgen05 with the partial top-k fused into the epilogue.
+//
+// Queries are the MMA M operand (128 per CTA), cache rows the N operand (256 per accumulator),
+// the embedding dimension is the K loop in 64-element (128-byte, swizzled) chunks.  With this
+// orientation tensor-memory lane i of an accumulator holds the scores of query i against 256
+// consecutive cache rows, so the epilogue thread that owns lane i owns query i: its admission
+// threshold stays in a register and a score costs one compare unless it enters the list.
+//
+// Warp roles (192 threads, one CTA per SM):
+//   warps 0-3  epilogue: tcgen05.ld the accumulator, filter against the per-query threshold,
+//              warp-cooperative sorted insert into per-query lists in shared memory
+//   warp 4     TMA producer: query chunk (16 KiB) + slab chunk (32 KiB) per ring stage
+//   warp 5     MMA issuer (one thread) and tensor-memory owner
+// Two 256-column accumulators alternate, so the epilogue of one row tile overlaps the MMAs
+// of the next.  CTA (p, t) scores query tile t against row tiles p, p + P, p + 2P, ...
+#include <math.h>
+
+#include "common.cuh"
+#include "kernels.h"
+#include "pipeline.cuh"
+
+namespace icc {
+
+constexpr int UM_THREADS = 192;
+constexpr int UM_QT = 128;            // queries per CTA (MMA M)
+constexpr int UM_RT = 256;            // cache rows per accumulator (MMA N)
+constexpr int UM_KC = 64;             // elements per K chunk (128 bytes)
+constexpr int UM_A_BYTES = UM_QT * UM_KC * 2;   // 16 KiB
+constexpr int UM_B_BYTES = UM_RT * UM_KC * 2;   // 32 KiB
+constexpr int UM_STAGE_BYTES = UM_A_BYTES + UM_B_BYTES;
+constexpr int UM_MAX_STAGES = 6;
+constexpr int UM_TMEM_COLS = 512;
+
+struct UmmaSmemTail {
+  uint64_t full[UM_MAX_STAGES];
+  uint64_t empty[UM_MAX_STAGES];
+  uint64_t acc_full[2];
+  uint64_t acc_empty[2];
+  uint64_t drain;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__global__ void __launch_bounds__(UM_THREADS, 1)
+umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_slab,
+                       int64_t n, int dim, int nq, int k, int n_query_tiles, int n_part, int n_stages,
+                       uint64_t* __restrict__ partials, int* dev_status) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  unsigned char* ring = smem;                                                        // n_stages * 48 KiB
+  uint64_t* lists = reinterpret_cast<uint64_t*>(ring + (size_t)n_stages * UM_STAGE_BYTES);  // [128][k]
+  UmmaSmemTail* tail = reinterpret_cast<UmmaSmemTail*>(lists + (size_t)UM_QT * k);
+  volatile int* abort_flag = &tail->abort_flag;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int qt = blockIdx.x % n_query_tiles;     // query tile of this CTA
+  const int part = blockIdx.x / n_query_tiles;   // row partition of this CTA
+  const int64_t n_tiles = (n + UM_RT - 1) / UM_RT;
+  const int n_kc = (dim + UM_KC - 1) / UM_KC;
+
+  if (tid == 0) {
+    for (int s = 0; s < n_stages; ++s) {
+      mbar_init(&tail->full[s], 1);
+      mbar_init(&tail->empty[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&tail->acc_full[b], 1);
+      mbar_init(&tail->acc_empty[b], 4);
+    }
+    mbar_init(&tail->drain, 1);
+    tail->abort_flag = 0;
+    mbar_fence_init();
+  }
+  for (int i = tid; i < UM_QT * k; i += UM_THREADS) lists[i] = KEY_EMPTY;
+  if (warp == 4 && lane == 0) {
+    prefetch_tmap(&tmap_q);
+    prefetch_tmap(&tmap_slab);
+  }
+  if (warp == 5) tmem_alloc(&tail->tmem_base, UM_TMEM_COLS);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = tail->tmem_base;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int64_t it = 0;
+      bool ok = true;
+      for (int64_t tile = part; tile < n_tiles && ok; tile += n_part) {
+        for (int kc = 0; kc < n_kc; ++kc, ++it) {
+          const int s = (int)(it % n_stages);
+          const uint32_t ph = (uint32_t)((it / n_stages) & 1);
+          ok = mbar_wait(&tail->empty[s], ph ^ 1u, abort_flag);
+          if (!ok) break;
+          unsigned char* a_dst = ring + (size_t)s * UM_STAGE_BYTES;
+          mbar_arrive_expect_tx(&tail->full[s], UM_STAGE_BYTES);
+          tma_load_2d(a_dst, &tmap_q, kc * UM_KC, qt * UM_QT, &tail->full[s]);
+          tma_load_2d(a_dst + UM_A_BYTES, &tmap_slab, kc * UM_KC, (int)(tile * UM_RT), &tail->full[s]);
+        }
+      }
+      if (!ok) {
+        report_status(dev_status, DEV_TIMEOUT_MBAR);
+        // loads already issued still write this CTA's shared memory: wait for them (bounded)
+        for (int64_t j = (it > n_stages ? it - n_stages : 0); j < it; ++j) {
+          const int s = (int)(j % n_stages);
+          const long long t0 = clock64();
+          while (!mbar_try_wait(&tail->full[s], (uint32_t)((j / n_stages) & 1)) &&
+                 clock64() - t0 < WAIT_LIMIT_CYCLES) {
+          }
+        }
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16_f32(UM_QT, UM_RT);
+      int64_t it = 0;
+      int64_t lt = 0;
+      bool ok = true;
+      for (int64_t tile = part; tile < n_tiles && ok; tile += n_part, ++lt) {
+        const int buf = (int)(lt & 1);
+        const uint32_t bph = (uint32_t)((lt >> 1) & 1);
+        ok = mbar_wait(&tail->acc_empty[buf], bph ^ 1u, abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * UM_RT);
+        for (int kc = 0; kc < n_kc; ++kc, ++it) {
+          const int s = (int)(it % n_stages);
+          const uint32_t ph = (uint32_t)((it / n_stages) & 1);
+          ok = mbar_wait(&tail->full[s], ph, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t a_addr = smem_u32(ring + (size_t)s * UM_STAGE_BYTES);
+          const uint64_t da = umma_desc_k_major_sw128(a_addr);
+          const uint64_t db = umma_desc_k_major_sw128(a_addr + UM_A_BYTES);
+#pragma unroll
+          for (int kk = 0; kk < UM_KC / 16; ++kk) {
+            // 16 bf16 = 32 bytes further along K inside the swizzled 128-byte row
+            umma_bf16(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (kc | kk) != 0 ? 1u : 0u);
+          }
+          umma_commit(&tail->empty[s]);   // stage reusable once these MMAs have read it
+        }
+        if (ok) umma_commit(&tail->acc_full[buf]);
+      }
+      // make sure nothing issued is still running before tensor memory is released
+      umma_commit(&tail->drain);
+      {
+        const long long t0 = clock64();
+        while (!mbar_try_wait(&tail->drain, 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {
+        }
+      }
+      if (!ok) report_status(dev_status, DEV_TIMEOUT_MBAR);
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 0-3)
+    const int q = qt * UM_QT + tid;                 // this thread's query (tensor-memory lane tid)
+    const bool real = q < nq;
+    uint64_t* warp_lists = lists + (size_t)(warp * 32) * k;
+    float thr_score = -INFINITY;                    // score of the k-th best so far
+    uint64_t thr_key = KEY_EMPTY;
+    int64_t lt = 0;
+    bool ok = true;
+    for (int64_t tile = part; tile < n_tiles; tile += n_part, ++lt) {
+      const int buf = (int)(lt & 1);
+      const uint32_t bph = (uint32_t)((lt >> 1) & 1);
+      ok = mbar_wait(&tail->acc_full[buf], bph, abort_flag);
+      ok = __all_sync(FULL_MASK, ok);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t t_addr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * UM_RT);
+      const int64_t row0 = tile * UM_RT;
+#pragma unroll 1
+      for (int cb = 0; cb < UM_RT / 32; ++cb) {
+        uint32_t v[32];
+        tmem_ld_32x32(t_addr + (uint32_t)(cb * 32), v);
+        tmem_ld_wait();
+        if (cb == UM_RT / 32 - 1) {
+          // the accumulator has been read completely: hand it back to the MMA issuer
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&tail->acc_empty[buf]);
+        }
+        const int64_t col0 = row0 + cb * 32;
+        if (col0 >= n) continue;                    // warp-uniform
+        uint32_t hitmask = 0;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) hitmask |= (__uint_as_float(v[c]) >= thr_score ? 1u : 0u) << c;
+        if (n - col0 < 32) hitmask &= (1u << (int)(n - col0)) - 1u;
+        if (!real) hitmask = 0;
+        if (!__any_sync(FULL_MASK, hitmask != 0)) continue;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const uint64_t key = make_key(__uint_as_float(v[c]), (uint32_t)(col0 + c));
+          unsigned hits = __ballot_sync(FULL_MASK, ((hitmask >> c) & 1u) && key > thr_key);
+          while (hits) {
+            const int src = __ffs(hits) - 1;
+            hits &= hits - 1;
+            const uint64_t hkey = __shfl_sync(FULL_MASK, key, src);
+            const uint64_t new_thr = warp_sorted_insert(warp_lists + (size_t)src * k, k, hkey, lane);
+            if (lane == src) {
+              thr_key = new_thr;
+              thr_score = (new_thr == KEY_EMPTY) ? -INFINITY : key_score(new_thr);
+            }
+          }
+        }
+      }
+    }
+    if (!ok && lane == 0) report_status(dev_status, DEV_TIMEOUT_MBAR);
+    __syncwarp();
+    // the 32 lists of this warp are contiguous both here and in the partials array
+    const int q_first = qt * UM_QT + warp * 32;
+    const int q_live = min(32, nq - q_first);
+    if (q_live > 0) {
+      uint64_t* dst = partials + ((size_t)part * nq + q_first) * k;
+      for (int i = lane; i < q_live * k; i += 32) dst[i] = warp_lists[i];
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, UM_TMEM_COLS);
+  }
+}
+
+cudaError_t umma_configure(int smem_optin) {
+  return cudaFuncSetAttribute(umma_score_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+}
+
+cudaError_t launch_umma(const UmmaParams& p, cudaStream_t st) {
+  if (p.n_stages < 2 || p.n_stages > UM_MAX_STAGES) return cudaErrorInvalidValue;
+  const size_t need = 1024 + (size_t)p.n_stages * UM_STAGE_BYTES + (size_t)UM_QT * p.k * 8 + sizeof(UmmaSmemTail);
+  if (need > (size_t)p.smem_bytes) return cudaErrorInvalidValue;
+  umma_score_topk_kernel<<<p.n_part * p.n_query_tiles, UM_THREADS, p.smem_bytes, st>>>(
+      p.tmap_q, p.tmap_slab, p.n, p.dim, p.nq, p.k, p.n_query_tiles, p.n_part, p.n_stages, p.partials,
+      p.dev_status);
+  return cudaGetLastError();
+}
+
+}  // namespace icc

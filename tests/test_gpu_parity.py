@@ -1,0 +1,210 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle element by
+element on the same seeded inputs.  Sizes span several tiles and ragged tails of every
+kernel path (scan pieces of 32 rows, tensor-core tiles of 256 rows x 128 queries x 64 dims)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2501_12689_b200 import (ICCache, ICCacheError, IC_PATH_AUTO, IC_PATH_GENERIC, IC_PATH_SCAN,
+                                   IC_PATH_UMMA, IC_ERR_FULL, IC_ERR_INVALID, workloads as wl)
+from parity_util import run_and_check, TOL
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+PATHS = {"auto": IC_PATH_AUTO, "generic": IC_PATH_GENERIC, "scan": IC_PATH_SCAN, "umma": IC_PATH_UMMA}
+
+
+def _gauss(n, dim, nq, seed, dtype="bf16"):
+    w = wl.Workload("g", n, dim, dtype, (nq,), 8, seed=seed)
+    return wl.cache_rows(w, DEV), wl.queries(w, nq, DEV)
+
+
+@pytest.mark.parametrize("path", ["generic", "scan", "umma", "auto"])
+def test_tiny_config(path):
+    w = wl.WORKLOADS["tiny"]
+    x, q = wl.cache_rows(w, DEV), wl.queries(w, 16, DEV)
+    run_and_check(x, q, w.k, path=PATHS[path], what=f"tiny/{path}")
+
+
+@pytest.mark.parametrize("path", ["generic", "scan", "umma", "auto"])
+@pytest.mark.parametrize("nq", [1, 4, 16, 64])
+def test_online_config_scaled(path, nq):
+    if path == "generic" and nq > 16:
+        pytest.skip("generic path is a slow cross-check; covered at nq <= 16")
+    w = wl.WORKLOADS["online"].scaled(70_001)      # 273.4 tensor-core tiles, 2187.5 scan pieces
+    x, q = wl.cache_rows(w, DEV), wl.queries(w, nq, DEV)
+    run_and_check(x, q, w.k, path=PATHS[path], what=f"online/{path}/nq{nq}")
+
+
+@pytest.mark.parametrize("path", ["scan", "umma"])
+@pytest.mark.parametrize("dim", [8, 40, 264, 520, 1024])
+def test_ragged_dims(path, dim):
+    x, q = _gauss(5_003, dim, 3, seed=20 + dim)
+    run_and_check(x, q, 5, path=PATHS[path], what=f"dim{dim}/{path}")
+
+
+@pytest.mark.parametrize("dim", [1032, 2048, 4096])
+def test_large_dims_take_the_tensor_core_path(dim):
+    x, q = _gauss(3_000, dim, 2, seed=30)
+    run_and_check(x, q, 4, path=IC_PATH_AUTO, what=f"dim{dim}/auto")
+    with ICCache(dim, 16) as c:
+        c.set_path(IC_PATH_SCAN)
+        c.insert(x[:16], wl.labels(16, DEV))
+        with pytest.raises(ICCacheError):
+            c.query(q, 2)
+
+
+@pytest.mark.parametrize("path", ["generic", "scan", "umma"])
+@pytest.mark.parametrize("n,k", [(1, 1), (5, 8), (31, 31), (300, 128), (4097, 64), (9, 128)])
+def test_small_caches_and_k_edges(path, n, k):
+    x, q = _gauss(n, 64, 3, seed=40 + n)
+    out_ids, out_scores, _ = run_and_check(x, q, k, path=PATHS[path], what=f"n{n}k{k}/{path}")
+    if k > n:
+        assert torch.all(out_ids[:, n:] == -1) and torch.all(torch.isneginf(out_scores[:, n:]))
+
+
+@pytest.mark.parametrize("path", ["generic", "scan", "umma"])
+def test_empty_cache(path):
+    with ICCache(64, 10) as c:
+        c.set_path(PATHS[path])
+        q = torch.randn(2, 64, device=DEV).to(torch.bfloat16)
+        ids, sc = c.query(q, 3)
+        c.sync()
+        assert torch.all(ids == -1) and torch.all(torch.isneginf(sc))
+        ids, sc = c.query(q[:0], 3)       # nq == 0 is a no-op
+        assert ids.shape == (0, 3)
+
+
+@pytest.mark.parametrize("path", ["scan", "umma"])
+@pytest.mark.parametrize("nq,k", [(2, 16), (130, 16), (257, 7)])
+def test_query_tiling(path, nq, k):
+    if path == "scan" and nq > 4:
+        nq = 7                                         # several scan passes with a ragged last one
+    x, q = _gauss(20_011, 128, nq, seed=50 + nq)
+    run_and_check(x, q, k, path=PATHS[path], what=f"qtile/{path}/nq{nq}")
+
+
+def test_more_queries_than_one_window():
+    x, q = _gauss(3_001, 64, 1030, seed=60)
+    run_and_check(x, q, 4, path=IC_PATH_UMMA, sample_queries=[0, 1, 127, 128, 1023, 1024, 1029], what="window")
+
+
+@pytest.mark.parametrize("path", ["generic", "scan", "umma"])
+def test_adversarial_orders(path):
+    # rows arrive in ascending order of their score against query 0: every row is a new best
+    dim, n = 64, 6_000
+    g = torch.Generator(device=DEV).manual_seed(70)
+    qv = torch.nn.functional.normalize(torch.randn(1, dim, generator=g, device=DEV), dim=1)
+    x = torch.nn.functional.normalize(torch.randn(n, dim, generator=g, device=DEV), dim=1).to(torch.bfloat16)
+    order = torch.argsort((x.float() @ qv.T).squeeze(1))
+    q = torch.cat([qv, -qv]).to(torch.bfloat16)       # second query sees descending order
+    run_and_check(x[order].contiguous(), q, 32, path=PATHS[path], what=f"ascending/{path}")
+    # all rows identical: every score ties, so the answer is the first k slots in order
+    same = x[:1].repeat(1000, 1).contiguous()
+    ids = wl.labels(1000, DEV)
+    out_ids, out_scores, _ = run_and_check(same, q[:1], 16, path=PATHS[path], ids=ids, what=f"ties/{path}")
+    assert torch.equal(out_ids[0], ids[:16].cpu())
+    assert torch.all(out_scores[0] == out_scores[0, 0])
+
+
+@pytest.mark.parametrize("path", ["scan", "umma"])
+def test_clustered_config_scaled_with_streaming_inserts(path):
+    w = wl.WORKLOADS["clustered"].scaled(60_000)
+    w = wl.Workload(**{**w.__dict__, "insert_rows": 1_000})
+    nq = 128 if path == "umma" else 4
+    x0 = wl.cache_rows(w, DEV)
+    cap = w.n + 3 * w.insert_rows
+    with ICCache(w.dim, cap) as c:
+        c.set_path(PATHS[path])
+        c.insert(x0, wl.labels(w.n, DEV))
+        allx = x0
+        for rnd in range(3):
+            new = wl.insert_batch(w, rnd, DEV)
+            c.insert(new, wl.labels(w.insert_rows, DEV, first_slot=allx.shape[0]))
+            allx = torch.cat([allx, new])
+            q = wl.queries(w, nq, DEV, round_idx=rnd, cache=allx)
+            ids, sc = c.query(q, w.k)
+            c.sync()
+            ref = oracle.search(wl.as_bits(allx), wl.as_bits(q), w.k, ids=wl.labels(allx.shape[0]).numpy(),
+                                want_all_scores=True)
+            lab = wl.labels(allx.shape[0]).numpy()
+            oracle.accept(ids.cpu().numpy(), sc.cpu().numpy(), ref["all_scores"], w.k, ids=lab, tol=1e-4,
+                          what=f"clustered/{path}/round{rnd}")
+            # planted queries copy rows inserted this round: they must come back first, score ~1
+            m = min(w.planted_queries, nq)
+            assert torch.all(sc[:m, 0] > 0.99)
+            assert torch.all(ids[:m, 0].cpu() >= 0)
+            # exact duplicates tie bit for bit: equal returned scores come back in slot order
+            sorter = np.argsort(lab)
+            slots = sorter[np.searchsorted(lab[sorter], ids.cpu().numpy())]
+            scn = sc.cpu().numpy()
+            tie = scn[:, 1:] == scn[:, :-1]
+            if nq >= 64:
+                assert tie.any(), "the workload should force exact score ties"
+            assert np.all(slots[:, 1:][tie] > slots[:, :-1][tie])
+
+
+@pytest.mark.parametrize("path", ["generic", "scan", "umma"])
+def test_split_inserts_equal_one_insert(path):
+    x, q = _gauss(10_000, 96, 4, seed=80)
+    a = run_and_check(x, q, 9, path=PATHS[path], what="one insert")
+    b = run_and_check(x, q, 9, path=PATHS[path], insert_splits=[1, 4_999, 5_000], what="three inserts")
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+@pytest.mark.parametrize("path", ["generic", "scan", "umma"])
+def test_fp32_input_with_normalisation(path):
+    g = torch.Generator(device=DEV).manual_seed(90)
+    x = torch.randn(8_000, 200, generator=g, device=DEV) * 3.0
+    x[17] = 0.0                                                   # a zero row stays zero
+    q = torch.randn(4, 200, generator=g, device=DEV) * 0.2
+    q[3] = x[4321] * 5.0                                          # same direction as a cached row
+    out_ids, out_scores, _ = run_and_check(x, q, 6, path=PATHS[path], normalize=True, what=f"normalize/{path}")
+    assert out_ids[3, 0].item() == wl.labels(8_000)[4321].item()
+    assert abs(out_scores[3, 0].item() - 1.0) < 5e-3
+
+
+def test_paths_agree_bit_for_bit_on_ids():
+    x, q = _gauss(40_000, 384, 4, seed=100)
+    res = {p: run_and_check(x, q, 10, path=PATHS[p], what=p)[:2] for p in ("generic", "scan", "umma")}
+    assert torch.equal(res["generic"][0], res["scan"][0])
+    assert torch.equal(res["generic"][0], res["umma"][0])
+    assert torch.allclose(res["generic"][1], res["umma"][1], atol=1e-5)
+
+
+def test_host_buffers_end_to_end():
+    x, q = _gauss(12_345, 128, 5, seed=110)
+    with ICCache(128, 12_345) as c:
+        c.insert_host(x.cpu(), wl.labels(12_345))
+        assert c.size == 12_345
+        ids_h, sc_h = c.query_host(q.cpu().pin_memory(), 7)
+        ids_d, sc_d = c.query(q, 7)
+        c.sync()
+        assert torch.equal(ids_h, ids_d.cpu()) and torch.equal(sc_h, sc_d.cpu())
+        assert c.launch_count > 0
+
+
+def test_error_returns_leave_the_cache_unchanged():
+    with ICCache(64, 100) as c:
+        x = torch.zeros(60, 64, device=DEV, dtype=torch.bfloat16)
+        ids = wl.labels(60, DEV)
+        c.insert(x, ids)
+        with pytest.raises(ICCacheError) as e:
+            c.insert(x, ids)
+        assert e.value.status == IC_ERR_FULL and c.size == 60
+        q = torch.zeros(1, 64, device=DEV, dtype=torch.bfloat16)
+        for bad_k in (0, 129):
+            with pytest.raises(ICCacheError) as e:
+                c.query(q, bad_k)
+            assert e.value.status == IC_ERR_INVALID
+        import paper_2501_12689_b200.binding as b
+        host_q = torch.zeros(1, 64, dtype=torch.bfloat16)
+        out_i = torch.empty(1, 4, dtype=torch.int64, device=DEV)
+        out_s = torch.empty(1, 4, dtype=torch.float32, device=DEV)
+        with pytest.raises(ICCacheError) as e:     # host pointer handed to the device entry point
+            b.ic_cache_query(c._h, host_q, 1, 4, out_i, out_s)
+        assert e.value.status == IC_ERR_INVALID
+    for dim, cap in ((0, 10), (12, 10), (8192, 10), (64, 0)):
+        with pytest.raises(ICCacheError):
+            ICCache(dim, cap)
