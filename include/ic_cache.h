@@ -89,7 +89,7 @@ typedef struct ic_cache_plan {
 /*
  * Create an empty cache for embeddings of `dim` components with room for `capacity` entries
  * on the current device, input dtype bf16, no normalisation, legacy default stream.
- * dim: multiple of 8, 8 <= dim <= IC_MAX_DIM.  capacity: 1 .. 2^32 - 2.
+ * dim: multiple of 8, 8 <= dim <= IC_MAX_DIM.  capacity: 1 .. 2^31 - 512.
  * Returns NULL on failure; ic_cache_last_error() then describes why.
  */
 ic_cache_t* ic_cache_create(int32_t dim, int64_t capacity);
@@ -156,6 +156,18 @@ int ic_cache_sync(ic_cache_t* c);
 
 /* Kernels launched by this handle so far (insert, query preparation, scoring, merge). */
 int64_t ic_cache_launch_count(const ic_cache_t* c);
+
+/*
+ * Measurement aid.  While enabled, every scoring-kernel launch and every merge launch of this
+ * handle is bracketed by a pair of CUDA events on the handle's stream (at most 16384 launches
+ * of each kind between two reads; later ones go unrecorded).
+ */
+int ic_cache_set_profiling(ic_cache_t* c, int32_t enable);
+
+/* Synchronise the stream and return the device time (ms) and number of the scoring and merge
+ * launches recorded since the previous read.  Any output pointer may be NULL. */
+int ic_cache_read_profile(ic_cache_t* c, double* scoring_ms, int64_t* scoring_launches,
+                          double* merge_ms, int64_t* merge_launches);
 
 /*
  * The launch plan the library would use for a query of nq vectors, k results, over n entries

@@ -71,6 +71,10 @@ SIGNATURES = {
     "ic_cache_clear": (ctypes.c_int, [ctypes.c_void_p]),
     "ic_cache_sync": (ctypes.c_int, [ctypes.c_void_p]),
     "ic_cache_launch_count": (ctypes.c_int64, [ctypes.c_void_p]),
+    "ic_cache_set_profiling": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32]),
+    "ic_cache_read_profile": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_double),
+                                             ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
+                                             ctypes.POINTER(ctypes.c_int64)]),
     "ic_cache_plan": (ctypes.c_int, [ctypes.c_int32, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                      ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ic_cache_plan_t)]),
     "ic_cache_last_error": (ctypes.c_char_p, []),
@@ -248,6 +252,18 @@ class ICCache:
 
     def sync(self) -> None:
         _check(load_library().ic_cache_sync(self._h))
+
+    def set_profiling(self, enable: bool) -> None:
+        _check(load_library().ic_cache_set_profiling(self._h, int(bool(enable))))
+
+    def read_profile(self) -> dict:
+        """Device time of the scoring and merge launches recorded since the last read."""
+        s_ms, m_ms = ctypes.c_double(), ctypes.c_double()
+        s_n, m_n = ctypes.c_int64(), ctypes.c_int64()
+        _check(load_library().ic_cache_read_profile(self._h, ctypes.byref(s_ms), ctypes.byref(s_n),
+                                                    ctypes.byref(m_ms), ctypes.byref(m_n)))
+        return {"scoring_ms": s_ms.value, "scoring_launches": s_n.value,
+                "merge_ms": m_ms.value, "merge_launches": m_n.value}
 
     @property
     def size(self) -> int:

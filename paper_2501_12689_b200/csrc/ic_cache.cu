@@ -9,6 +9,7 @@
 
 #include <algorithm>
 #include <new>
+#include <vector>
 
 #include "../../include/ic_cache.h"
 #include "kernels.h"
@@ -80,6 +81,10 @@ struct ic_cache {
   EncodeTiledFn encode = nullptr;
   CUtensorMap tmap_slab;
   bool have_tmap_slab = false;
+  // optional per-kernel timing (ic_cache_set_profiling)
+  bool profiling = false;
+  std::vector<cudaEvent_t> ev_score, ev_merge;   // start/stop pairs
+  size_t n_ev_score = 0, n_ev_merge = 0;         // events used since the last read
 };
 
 namespace {
@@ -182,6 +187,22 @@ int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32
   return IC_OK;
 }
 
+constexpr size_t MAX_PROFILE_EVENTS = 2 * 16384;
+
+// Record one event of a start/stop pair; silently stops recording when the pool is full.
+void profile_mark(ic_cache* c, std::vector<cudaEvent_t>& pool, size_t& used) {
+  if (!c->profiling || used >= MAX_PROFILE_EVENTS) return;
+  if (used == pool.size()) {
+    cudaEvent_t ev;
+    if (cudaEventCreate(&ev) != cudaSuccess) {
+      cudaGetLastError();
+      return;
+    }
+    pool.push_back(ev);
+  }
+  cudaEventRecord(pool[used++], c->stream);
+}
+
 int check_timeout(ic_cache* c) {
   if (c->h_status && *reinterpret_cast<volatile int*>(c->h_status) != 0)
     return fail(IC_ERR_TIMEOUT, "an earlier kernel gave up on a bounded wait (code %d); call ic_cache_sync to clear", *c->h_status);
@@ -216,6 +237,7 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
   c->launches += 1;
   uint64_t* partials = static_cast<uint64_t*>(c->partials.p);
 
+  profile_mark(c, c->ev_score, c->n_ev_score);
   if (pl.path == IC_PATH_GENERIC) {
     for (int q0 = 0; q0 < nq; q0 += GENERIC_QB) {
       e = icc::launch_generic(c->slab, c->size, c->dim, static_cast<const float*>(c->q_f32.p), q0, nq, k,
@@ -264,9 +286,12 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
     if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core scoring launch failed: %s", cudaGetErrorString(e));
     c->launches += 1;
   }
+  profile_mark(c, c->ev_score, c->n_ev_score);
+  profile_mark(c, c->ev_merge, c->n_ev_merge);
   e = icc::launch_merge(partials, pl.n_partitions, nq, k, c->ids, out_ids, out_scores, c->stream);
   if (e != cudaSuccess) return fail(IC_ERR_CUDA, "merge launch failed: %s", cudaGetErrorString(e));
   c->launches += 1;
+  profile_mark(c, c->ev_merge, c->n_ev_merge);
   return IC_OK;
 }
 
@@ -299,8 +324,8 @@ ic_cache_t* ic_cache_create_ex(int32_t dim, int64_t capacity, const ic_cache_opt
     fail(IC_ERR_INVALID, "dim %d must be a multiple of 8 in [8, %d]", dim, IC_MAX_DIM);
     return nullptr;
   }
-  if (capacity < 1 || capacity > 0xfffffffell) {
-    fail(IC_ERR_INVALID, "capacity %lld outside [1, 2^32-2]", (long long)capacity);
+  if (capacity < 1 || capacity > 0x7fffffffll - 511) {
+    fail(IC_ERR_INVALID, "capacity %lld outside [1, 2^31-512]", (long long)capacity);
     return nullptr;
   }
   ic_cache_opts_t o;
@@ -452,6 +477,8 @@ void ic_cache_destroy(ic_cache_t* c) {
   release(c->stage_ids);
   release(c->stage_scores);
   if (c->h_status) cudaFreeHost(c->h_status);
+  for (cudaEvent_t ev : c->ev_score) cudaEventDestroy(ev);
+  for (cudaEvent_t ev : c->ev_merge) cudaEventDestroy(ev);
   cudaGetLastError();
   delete c;
 }
@@ -593,6 +620,41 @@ int ic_cache_sync(ic_cache_t* c) {
     *c->h_status = 0;
     return fail(IC_ERR_TIMEOUT, "a kernel gave up on a bounded wait (code %d); its results are incomplete", code);
   }
+  return IC_OK;
+}
+
+int ic_cache_set_profiling(ic_cache_t* c, int32_t enable) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  c->profiling = enable != 0;
+  return IC_OK;
+}
+
+int ic_cache_read_profile(ic_cache_t* c, double* scoring_ms, int64_t* scoring_launches, double* merge_ms,
+                          int64_t* merge_launches) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  DeviceGuard guard(c->device);
+  cudaError_t e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "stream sync failed: %s", cudaGetErrorString(e));
+  double sums[2] = {0.0, 0.0};
+  int64_t counts[2] = {0, 0};
+  std::vector<cudaEvent_t>* pools[2] = {&c->ev_score, &c->ev_merge};
+  size_t* used[2] = {&c->n_ev_score, &c->n_ev_merge};
+  for (int w = 0; w < 2; ++w) {
+    for (size_t i = 0; i + 1 < *used[w]; i += 2) {
+      float ms = 0.0f;
+      if (cudaEventElapsedTime(&ms, (*pools[w])[i], (*pools[w])[i + 1]) == cudaSuccess) {
+        sums[w] += ms;
+        counts[w] += 1;
+      } else {
+        cudaGetLastError();
+      }
+    }
+    *used[w] = 0;
+  }
+  if (scoring_ms) *scoring_ms = sums[0];
+  if (scoring_launches) *scoring_launches = counts[0];
+  if (merge_ms) *merge_ms = sums[1];
+  if (merge_launches) *merge_launches = counts[1];
   return IC_OK;
 }
 
