@@ -1,0 +1,112 @@
+"""CPU-only checks: the shared library loads and exports every symbol the header declares,
+argument validation and launch planning work without a GPU, and the benchmark's cross-rank
+aggregation is right on a two-process gloo group."""
+import json
+import os
+import re
+import subprocess
+import sys
+
+import pytest
+
+import paper_2501_12689_b200 as pkg
+from paper_2501_12689_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "ic_cache.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ic_cache_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2501_12689_b200.build import build
+    build()
+    lib = pkg.load_library()
+    names = _declared_symbols()
+    assert "ic_cache_create" in names and "ic_cache_query" in names and len(names) >= 15
+    for name in names:
+        assert hasattr(lib, name), f"{name} is declared in ic_cache.h but not exported"
+        assert name in binding.SIGNATURES, f"{name} has no Python binding signature"
+    assert lib.ic_cache_version() >= 100
+
+
+def test_header_constants_match_binding():
+    text = open(os.path.join(ROOT, "include", "ic_cache.h")).read()
+    assert int(re.search(r"#define IC_MAX_K (\d+)", text).group(1)) == binding.IC_MAX_K
+    assert int(re.search(r"#define IC_MAX_DIM (\d+)", text).group(1)) == binding.IC_MAX_DIM
+    for name in ("IC_ERR_INVALID", "IC_ERR_NOMEM", "IC_ERR_FULL", "IC_ERR_CUDA", "IC_ERR_UNSUPPORTED", "IC_ERR_TIMEOUT"):
+        assert int(re.search(name + r" = (-\d+)", text).group(1)) == getattr(binding, name)
+
+
+def test_plan_paths_and_shapes():
+    p = pkg.ic_cache_plan(768, 1_000_000, 1, 10)
+    assert p["path"] == pkg.IC_PATH_SCAN and p["query_tile"] == 1 and p["n_ctas"] == 148 and p["n_stages"] >= 2
+    p = pkg.ic_cache_plan(768, 1_000_000, 4, 10)
+    assert p["path"] == pkg.IC_PATH_SCAN and p["query_tile"] == 4 and p["n_launches"] == 1
+    p = pkg.ic_cache_plan(768, 1_000_000, 64, 10)
+    assert p["path"] == pkg.IC_PATH_UMMA and p["n_query_tiles"] == 1 and p["n_partitions"] == 148
+    p = pkg.ic_cache_plan(1024, 4_000_000, 256, 32)
+    assert p["n_query_tiles"] == 2 and p["n_partitions"] == 74 and p["n_ctas"] == 148
+    p = pkg.ic_cache_plan(768, 16_000_000, 1024, 64)
+    assert p["n_query_tiles"] == 8 and p["n_partitions"] == 18 and p["n_ctas"] == 144 and p["n_launches"] == 1
+    assert p["smem_bytes"] <= 232448
+    p = pkg.ic_cache_plan(768, 16_000_000, 3000, 64)
+    assert p["n_launches"] == 3
+    p = pkg.ic_cache_plan(2048, 1000, 2, 5)          # too wide for the scan path
+    assert p["path"] == pkg.IC_PATH_UMMA
+    p = pkg.ic_cache_plan(64, 1000, 6, 128, path=pkg.IC_PATH_GENERIC)
+    assert p["n_launches"] == 2 and p["n_partitions"] * 128 * 8 < 232448
+    for k in (1, 10, 64, 128):                       # every k leaves at least two ring stages
+        assert pkg.ic_cache_plan(4096, 10, 128, k)["n_stages"] >= 2
+
+
+@pytest.mark.parametrize("args", [
+    dict(dim=12, n=10, nq=1, k=1), dict(dim=0, n=10, nq=1, k=1), dict(dim=8192, n=10, nq=1, k=1),
+    dict(dim=64, n=10, nq=0, k=1), dict(dim=64, n=10, nq=1, k=0), dict(dim=64, n=10, nq=1, k=129),
+    dict(dim=64, n=-1, nq=1, k=1), dict(dim=64, n=10, nq=1, k=1, path=9),
+])
+def test_plan_rejects_bad_arguments(args):
+    with pytest.raises(pkg.ICCacheError) as e:
+        pkg.ic_cache_plan(**args)
+    assert e.value.status == pkg.IC_ERR_INVALID and str(e.value)
+
+
+def test_forced_scan_path_rejects_wide_rows():
+    with pytest.raises(pkg.ICCacheError) as e:
+        pkg.ic_cache_plan(2048, 10, 1, 1, path=pkg.IC_PATH_SCAN)
+    assert e.value.status == pkg.IC_ERR_UNSUPPORTED
+
+
+def test_create_fails_loudly_without_a_gpu_or_with_bad_arguments():
+    import torch
+    lib = pkg.load_library()
+    assert not lib.ic_cache_create(12, 10) and b"multiple of 8" in lib.ic_cache_last_error()
+    assert not lib.ic_cache_create(64, 0) and b"capacity" in lib.ic_cache_last_error()
+    if not torch.cuda.is_available():
+        assert not lib.ic_cache_create(64, 10)
+        assert b"no CPU fallback" in lib.ic_cache_last_error()
+    # NULL handles are rejected, destroy(NULL) is a no-op
+    assert lib.ic_cache_size(None) == pkg.IC_ERR_INVALID
+    assert lib.ic_cache_insert(None, None, None, 1) == pkg.IC_ERR_INVALID
+    assert lib.ic_cache_query(None, None, 1, 1, None, None) == pkg.IC_ERR_INVALID
+    lib.ic_cache_destroy(None)
+
+
+def test_two_rank_gloo_aggregation():
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+           "--master-addr", "127.0.0.1", "--master-port", "29531", os.path.join(ROOT, "tests", "_gloo_worker.py")]
+    r = subprocess.run(cmd, capture_output=True, text=True, timeout=240, cwd=ROOT)
+    assert r.returncode == 0, r.stdout + r.stderr
+    assert "AGGREGATE_OK 15.0 3000.0" in r.stdout
+
+
+def test_reference_arm_runs_the_oracle_and_prints_the_contract_line():
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiny",
+                        "--steps", "2", "--warmup", "1"], capture_output=True, text=True, timeout=240, cwd=ROOT)
+    assert r.returncode == 0, r.stderr
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["unit"] == "queries/s" and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
