@@ -9,7 +9,7 @@
 
 namespace icc {
 
-constexpr int MERGE_THREADS = 128;
+constexpr int MERGE_THREADS = 256;
 
 __global__ void __launch_bounds__(MERGE_THREADS)
 merge_topk_kernel(const uint64_t* __restrict__ partials, int n_part, int nq, int k,
@@ -23,9 +23,12 @@ merge_topk_kernel(const uint64_t* __restrict__ partials, int n_part, int nq, int
 
   const int q = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
   const int total = n_part * k;
+  // list p of this query is k contiguous keys at partials[(p * nq + q) * k]; several loads
+  // per thread are in flight at once
+#pragma unroll 4
   for (int i = tid; i < total; i += MERGE_THREADS) {
     const int p = i / k, j = i - p * k;
-    cand[i] = partials[((size_t)p * nq + q) * k + j];
+    cand[i] = __ldg(partials + ((size_t)p * nq + q) * k + j);
   }
   for (int p = tid; p < n_part; p += MERGE_THREADS) pos[p] = 0;
   __syncthreads();

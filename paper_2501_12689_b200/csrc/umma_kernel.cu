@@ -8,7 +8,7 @@
 //
 // Warp roles (192 threads, one CTA per SM):
 //   warps 0-3  epilogue: tcgen05.ld the accumulator, filter against the per-query threshold,
-//              warp-cooperative sorted insert into per-query lists in shared memory
+//              admit the rare survivors into per-query lists in shared memory
 //   warp 4     TMA producer: query chunk (16 KiB) + slab chunk (32 KiB) per ring stage
 //   warp 5     MMA issuer (one thread) and tensor-memory owner
 // Two 256-column accumulators alternate, so the epilogue of one row tile overlaps the MMAs
@@ -154,11 +154,19 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     }
   } else {
     // ------------------------------------------------------------ epilogue (warps 0-3)
-    const int q = qt * UM_QT + tid;                 // this thread's query (tensor-memory lane tid)
+    // Thread t owns query qt*128 + t (tensor-memory lane t).  Its k best candidates live in an
+    // unsorted private list in shared memory, stored transposed ([k][32] per warp) so that the
+    // 32 lanes of a warp touch 32 consecutive 8-byte words.  The admission threshold (smallest
+    // key of the list, its score and its position) stays in registers; admitting a candidate
+    // overwrites the smallest entry and rescans the k entries for the new smallest.  Lanes
+    // admit in parallel, each into its own list, so no warp-level synchronisation is needed.
+    const int q = qt * UM_QT + tid;
     const bool real = q < nq;
     uint64_t* warp_lists = lists + (size_t)(warp * 32) * k;
-    float thr_score = -INFINITY;                    // score of the k-th best so far
+    uint64_t* my_list = warp_lists + lane;           // entry i at my_list[i * 32]
+    float thr_score = real ? -INFINITY : __int_as_float(0x7fc00000);   // NaN never admits
     uint64_t thr_key = KEY_EMPTY;
+    int min_pos = 0;
     int64_t lt = 0;
     bool ok = true;
     for (int64_t tile = part; tile < n_tiles; tile += n_part, ++lt) {
@@ -183,37 +191,58 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         }
         const int64_t col0 = row0 + cb * 32;
         if (col0 >= n) continue;                    // warp-uniform
-        uint32_t hitmask = 0;
+        if (n - col0 < 32) {                        // ragged last tile: columns past n never admit
 #pragma unroll
-        for (int c = 0; c < 32; ++c) hitmask |= (__uint_as_float(v[c]) >= thr_score ? 1u : 0u) << c;
-        if (n - col0 < 32) hitmask &= (1u << (int)(n - col0)) - 1u;
-        if (!real) hitmask = 0;
-        if (!__any_sync(FULL_MASK, hitmask != 0)) continue;
+          for (int c = 0; c < 32; ++c)
+            if (col0 + c >= n) v[c] = 0x7fc00000u;
+        }
+        float best = __uint_as_float(v[0]);
+#pragma unroll
+        for (int c = 1; c < 32; ++c) best = fmaxf(best, __uint_as_float(v[c]));
+        if (!(best >= thr_score)) continue;         // common case: nothing beats the threshold
 #pragma unroll
         for (int c = 0; c < 32; ++c) {
-          const uint64_t key = make_key(__uint_as_float(v[c]), (uint32_t)(col0 + c));
-          unsigned hits = __ballot_sync(FULL_MASK, ((hitmask >> c) & 1u) && key > thr_key);
-          while (hits) {
-            const int src = __ffs(hits) - 1;
-            hits &= hits - 1;
-            const uint64_t hkey = __shfl_sync(FULL_MASK, key, src);
-            const uint64_t new_thr = warp_sorted_insert(warp_lists + (size_t)src * k, k, hkey, lane);
-            if (lane == src) {
-              thr_key = new_thr;
-              thr_score = (new_thr == KEY_EMPTY) ? -INFINITY : key_score(new_thr);
+          const float s = __uint_as_float(v[c]);
+          if (s >= thr_score) {
+            const uint64_t key = make_key(s, (uint32_t)(col0 + c));
+            if (key > thr_key) {
+              my_list[min_pos * 32] = key;
+              uint64_t m = ~0ull;
+              int mp = 0;
+#pragma unroll 4
+              for (int i = 0; i < k; ++i) {
+                const uint64_t e = my_list[i * 32];
+                if (e < m) { m = e; mp = i; }
+              }
+              thr_key = m;
+              min_pos = mp;
+              thr_score = (m == KEY_EMPTY) ? -INFINITY : key_score(m);
             }
           }
         }
       }
     }
     if (!ok && lane == 0) report_status(dev_status, DEV_TIMEOUT_MBAR);
+    // sort each private list descending (insertion sort, lanes in parallel)
+    for (int i = 1; i < k; ++i) {
+      const uint64_t e = my_list[i * 32];
+      int j = i - 1;
+      while (j >= 0 && my_list[j * 32] < e) {
+        my_list[(j + 1) * 32] = my_list[j * 32];
+        --j;
+      }
+      my_list[(j + 1) * 32] = e;
+    }
     __syncwarp();
-    // the 32 lists of this warp are contiguous both here and in the partials array
+    // transpose out: the partial lists of this warp's queries are contiguous in global memory
     const int q_first = qt * UM_QT + warp * 32;
     const int q_live = min(32, nq - q_first);
     if (q_live > 0) {
       uint64_t* dst = partials + ((size_t)part * nq + q_first) * k;
-      for (int i = lane; i < q_live * k; i += 32) dst[i] = warp_lists[i];
+      for (int i = lane; i < q_live * k; i += 32) {
+        const int ql = i / k, e = i - ql * k;
+        dst[i] = warp_lists[e * 32 + ql];
+      }
     }
   }
   tc_fence_before_sync();
