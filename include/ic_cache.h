@@ -84,6 +84,7 @@ typedef struct ic_cache_plan {
   int32_t n_stages;      /* shared-memory ring stages (0 for the generic path)             */
   int32_t smem_bytes;    /* dynamic shared memory of the scoring kernel                    */
   int32_t n_launches;    /* scoring launches needed for the whole batch                    */
+  int32_t queue_cap;     /* tensor-core path: candidate queue entries per query (else 0)   */
 } ic_cache_plan_t;
 
 /*

@@ -178,7 +178,12 @@ int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32
     out->n_query_tiles = (window + QUERY_TILE - 1) / QUERY_TILE;
     out->n_partitions = std::max(1, std::min(sm_count / out->n_query_tiles, merge_lists_max));
     out->n_ctas = out->n_partitions * out->n_query_tiles;
-    const int fixed = 2048 + QUERY_TILE * k * 8;   // 1 KiB alignment slack + barriers, lists
+    // 1 KiB alignment slack + 256 B of barriers, the per-query lists, then as many candidate
+    // queue entries per query (up to 8) as still leave room for two ring stages
+    const int base = 1024 + 256 + QUERY_TILE * k * 8;
+    out->queue_cap = std::min(8, (smem_optin - base - 2 * UMMA_STAGE_BYTES) / (QUERY_TILE * 8));
+    if (out->queue_cap < 1) return fail(IC_ERR_UNSUPPORTED, "tensor-core path: shared memory too small");
+    const int fixed = base + QUERY_TILE * out->queue_cap * 8;
     out->n_stages = std::min(6, (smem_optin - fixed) / UMMA_STAGE_BYTES);
     if (out->n_stages < 2) return fail(IC_ERR_UNSUPPORTED, "tensor-core path: shared memory too small");
     out->smem_bytes = fixed + out->n_stages * UMMA_STAGE_BYTES;
@@ -279,6 +284,7 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
     up.n_query_tiles = pl.n_query_tiles;
     up.n_part = pl.n_partitions;
     up.n_stages = pl.n_stages;
+    up.queue_cap = pl.queue_cap;
     up.smem_bytes = pl.smem_bytes;
     up.partials = partials;
     up.dev_status = c->d_status;

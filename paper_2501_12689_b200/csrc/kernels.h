@@ -45,6 +45,7 @@ struct UmmaParams {
   int n_query_tiles;
   int n_part;
   int n_stages;
+  int queue_cap;          // per-query candidate queue entries in shared memory
   int smem_bytes;
   uint64_t* partials;     // [n_part][nq][k]
   int* dev_status;

@@ -43,13 +43,14 @@ struct UmmaSmemTail {
 
 __global__ void __launch_bounds__(UM_THREADS, 1)
 umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_slab,
-                       int64_t n, int dim, int nq, int k, int n_query_tiles, int n_part, int n_stages,
+                       int64_t n, int dim, int nq, int k, int n_query_tiles, int n_part, int n_stages, int qcap,
                        uint64_t* __restrict__ partials, int* dev_status) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   unsigned char* ring = smem;                                                        // n_stages * 48 KiB
   uint64_t* lists = reinterpret_cast<uint64_t*>(ring + (size_t)n_stages * UM_STAGE_BYTES);  // [128][k]
-  UmmaSmemTail* tail = reinterpret_cast<UmmaSmemTail*>(lists + (size_t)UM_QT * k);
+  uint64_t* queues = lists + (size_t)UM_QT * k;                                      // [128][qcap]
+  UmmaSmemTail* tail = reinterpret_cast<UmmaSmemTail*>(queues + (size_t)UM_QT * qcap);
   volatile int* abort_flag = &tail->abort_flag;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -157,16 +158,40 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     // Thread t owns query qt*128 + t (tensor-memory lane t).  Its k best candidates live in an
     // unsorted private list in shared memory, stored transposed ([k][32] per warp) so that the
     // 32 lanes of a warp touch 32 consecutive 8-byte words.  The admission threshold (smallest
-    // key of the list, its score and its position) stays in registers; admitting a candidate
-    // overwrites the smallest entry and rescans the k entries for the new smallest.  Lanes
-    // admit in parallel, each into its own list, so no warp-level synchronisation is needed.
+    // key of the list, its score and its position) stays in registers.
+    // A score that passes the threshold is only appended to the thread's small queue (cheap,
+    // so lanes that hit in different columns cost little when the warp serialises them); the
+    // queues are drained with all lanes working on their own list at the same time: admitting
+    // a candidate overwrites the list's smallest entry and rescans the k entries for the new
+    // smallest.
     const int q = qt * UM_QT + tid;
     const bool real = q < nq;
     uint64_t* warp_lists = lists + (size_t)(warp * 32) * k;
-    uint64_t* my_list = warp_lists + lane;           // entry i at my_list[i * 32]
+    uint64_t* my_list = warp_lists + lane;                              // entry i at my_list[i * 32]
+    uint64_t* my_queue = queues + (size_t)(warp * 32) * qcap + lane;    // entry i at my_queue[i * 32]
     float thr_score = real ? -INFINITY : __int_as_float(0x7fc00000);   // NaN never admits
     uint64_t thr_key = KEY_EMPTY;
     int min_pos = 0;
+    int cnt = 0;
+    auto drain = [&]() {
+      for (int i = 0; i < cnt; ++i) {
+        const uint64_t key = my_queue[i * 32];
+        if (key > thr_key) {
+          my_list[min_pos * 32] = key;
+          uint64_t m = ~0ull;
+          int mp = 0;
+#pragma unroll 4
+          for (int j = 0; j < k; ++j) {
+            const uint64_t e = my_list[j * 32];
+            if (e < m) { m = e; mp = j; }
+          }
+          thr_key = m;
+          min_pos = mp;
+          thr_score = (m == KEY_EMPTY) ? -INFINITY : key_score(m);
+        }
+      }
+      cnt = 0;
+    };
     int64_t lt = 0;
     bool ok = true;
     for (int64_t tile = part; tile < n_tiles; tile += n_part, ++lt) {
@@ -199,28 +224,19 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         float best = __uint_as_float(v[0]);
 #pragma unroll
         for (int c = 1; c < 32; ++c) best = fmaxf(best, __uint_as_float(v[c]));
-        if (!(best >= thr_score)) continue;         // common case: nothing beats the threshold
+        if (!__any_sync(FULL_MASK, best >= thr_score)) continue;   // common case: nothing passes
 #pragma unroll
         for (int c = 0; c < 32; ++c) {
           const float s = __uint_as_float(v[c]);
           if (s >= thr_score) {
-            const uint64_t key = make_key(s, (uint32_t)(col0 + c));
-            if (key > thr_key) {
-              my_list[min_pos * 32] = key;
-              uint64_t m = ~0ull;
-              int mp = 0;
-#pragma unroll 4
-              for (int i = 0; i < k; ++i) {
-                const uint64_t e = my_list[i * 32];
-                if (e < m) { m = e; mp = i; }
-              }
-              thr_key = m;
-              min_pos = mp;
-              thr_score = (m == KEY_EMPTY) ? -INFINITY : key_score(m);
-            }
+            if (cnt == qcap) drain();
+            my_queue[cnt * 32] = make_key(s, (uint32_t)(col0 + c));
+            ++cnt;
           }
         }
+        if (__any_sync(FULL_MASK, 2 * cnt >= qcap)) drain();
       }
+      drain();   // fresh thresholds for the next tile
     }
     if (!ok && lane == 0) report_status(dev_status, DEV_TIMEOUT_MBAR);
     // sort each private list descending (insertion sort, lanes in parallel)
@@ -259,10 +275,11 @@ cudaError_t umma_configure(int smem_optin) {
 
 cudaError_t launch_umma(const UmmaParams& p, cudaStream_t st) {
   if (p.n_stages < 2 || p.n_stages > UM_MAX_STAGES) return cudaErrorInvalidValue;
-  const size_t need = 1024 + (size_t)p.n_stages * UM_STAGE_BYTES + (size_t)UM_QT * p.k * 8 + sizeof(UmmaSmemTail);
+  if (p.queue_cap < 1) return cudaErrorInvalidValue;
+  const size_t need = 1024 + (size_t)p.n_stages * UM_STAGE_BYTES + (size_t)UM_QT * (p.k + p.queue_cap) * 8 + sizeof(UmmaSmemTail);
   if (need > (size_t)p.smem_bytes) return cudaErrorInvalidValue;
   umma_score_topk_kernel<<<p.n_part * p.n_query_tiles, UM_THREADS, p.smem_bytes, st>>>(
-      p.tmap_q, p.tmap_slab, p.n, p.dim, p.nq, p.k, p.n_query_tiles, p.n_part, p.n_stages, p.partials,
+      p.tmap_q, p.tmap_slab, p.n, p.dim, p.nq, p.k, p.n_query_tiles, p.n_part, p.n_stages, p.queue_cap, p.partials,
       p.dev_status);
   return cudaGetLastError();
 }
