@@ -85,6 +85,8 @@ typedef struct ic_cache_plan {
   int32_t smem_bytes;    /* dynamic shared memory of the scoring kernel                    */
   int32_t n_launches;    /* scoring launches needed for the whole batch                    */
   int32_t queue_cap;     /* tensor-core path: candidate queue entries per query (else 0)   */
+  int32_t seed_tiles;    /* tensor-core path: 256-row tiles scored first to seed the
+                            per-query thresholds of the main pass (0 = single pass)        */
 } ic_cache_plan_t;
 
 /*

@@ -35,6 +35,8 @@ constexpr int SCAN_MAX_Q = 4;
 constexpr int SCAN_MAX_DIM = 1024;
 constexpr int SCAN_ROWS_PER_STAGE = 32;
 constexpr int GENERIC_QB = 4;
+constexpr int SEED_MIN_TILES_PER_CTA = 8;  // tcgen05 path: seed thresholds when a CTA has this many tiles
+constexpr int SEED_FRACTION = 16;          // share of the row tiles scored by the seeding pass
 
 struct DeviceGuard {
   int prev = -1;
@@ -74,7 +76,7 @@ struct ic_cache {
   bool own_slab = false;
   int64_t* ids = nullptr;
   bool own_ids = false;
-  Buffer q_bf16, q_f32, partials, stage_in, stage_ids, stage_scores;
+  Buffer q_bf16, q_f32, partials, thr, stage_in, stage_ids, stage_scores;
   int* h_status = nullptr;  // pinned, mapped; kernels write a code when a bounded wait expires
   int* d_status = nullptr;
   int64_t launches = 0;
@@ -176,8 +178,15 @@ int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32
   } else {
     out->query_tile = QUERY_TILE;
     out->n_query_tiles = (window + QUERY_TILE - 1) / QUERY_TILE;
-    out->n_partitions = std::max(1, std::min(sm_count / out->n_query_tiles, merge_lists_max));
+    out->n_partitions = std::max(1, std::min(sm_count / out->n_query_tiles, merge_lists_max - 1));
     out->n_ctas = out->n_partitions * out->n_query_tiles;
+    // Threshold seeding: with enough row tiles per CTA, first score 1/16 of them, merge that
+    // sample's lists into its exact top-k and start the main pass from the sample's k-th key.
+    const int64_t n_tiles = (n + ROW_TILE - 1) / ROW_TILE;
+    if (n_tiles >= (int64_t)SEED_MIN_TILES_PER_CTA * out->n_partitions) {
+      const int64_t t = n_tiles / SEED_FRACTION / out->n_partitions * out->n_partitions;
+      out->seed_tiles = (int32_t)std::max<int64_t>(out->n_partitions, t);
+    }
     // 1 KiB alignment slack + 256 B of barriers, the per-query lists, then as many candidate
     // queue entries per query (up to 8) as still leave room for two ring stages
     const int base = 1024 + 256 + QUERY_TILE * k * 8;
@@ -187,7 +196,7 @@ int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32
     out->n_stages = std::min(6, (smem_optin - fixed) / UMMA_STAGE_BYTES);
     if (out->n_stages < 2) return fail(IC_ERR_UNSUPPORTED, "tensor-core path: shared memory too small");
     out->smem_bytes = fixed + out->n_stages * UMMA_STAGE_BYTES;
-    out->n_launches = n_windows;
+    out->n_launches = n_windows * (out->seed_tiles > 0 ? 2 : 1);
   }
   return IC_OK;
 }
@@ -234,13 +243,17 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
   const int nq_pad = (nq + QUERY_TILE - 1) / QUERY_TILE * QUERY_TILE;
   if ((rc = ensure(c, c->q_bf16, (size_t)nq_pad * c->dim * 2, "query staging (bf16)")) != IC_OK) return rc;
   if ((rc = ensure(c, c->q_f32, (size_t)nq * c->dim * 4, "query staging (fp32)")) != IC_OK) return rc;
-  if ((rc = ensure(c, c->partials, (size_t)pl.n_partitions * nq * k * 8, "partial top-k lists")) != IC_OK) return rc;
+  // lists of the main pass, one merged list of the seeding pass, lists of the seeding pass
+  const size_t list_block = (size_t)nq * k;   // keys of one partition
+  if ((rc = ensure(c, c->partials, (size_t)(2 * pl.n_partitions + 1) * list_block * 8, "partial top-k lists")) != IC_OK) return rc;
+  if ((rc = ensure(c, c->thr, (size_t)nq * 8, "seed thresholds")) != IC_OK) return rc;
 
   cudaError_t e = icc::launch_convert_rows(q, c->input_dtype == IC_F32, nq, c->dim, c->normalize, c->q_bf16.p,
                                            static_cast<float*>(c->q_f32.p), nq_pad, c->stream);
   if (e != cudaSuccess) return fail(IC_ERR_CUDA, "query preparation launch failed: %s", cudaGetErrorString(e));
   c->launches += 1;
   uint64_t* partials = static_cast<uint64_t*>(c->partials.p);
+  int n_final_lists = pl.n_partitions;
 
   profile_mark(c, c->ev_score, c->n_ev_score);
   if (pl.path == IC_PATH_GENERIC) {
@@ -286,15 +299,36 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
     up.n_stages = pl.n_stages;
     up.queue_cap = pl.queue_cap;
     up.smem_bytes = pl.smem_bytes;
-    up.partials = partials;
     up.dev_status = c->d_status;
+    const int64_t n_tiles = (c->size + ROW_TILE - 1) / ROW_TILE;
+    if (pl.seed_tiles > 0) {
+      // seeding pass over the first seed_tiles row tiles -> lists behind the main pass's
+      uint64_t* seed_lists = partials + (size_t)(pl.n_partitions + 1) * list_block;
+      up.tile_begin = 0;
+      up.tile_end = pl.seed_tiles;
+      up.thr_floor = nullptr;
+      up.partials = seed_lists;
+      e = icc::launch_umma(up, c->stream);
+      if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core seeding launch failed: %s", cudaGetErrorString(e));
+      c->launches += 1;
+      // exact top-k of the sample, kept as list number n_partitions of the final merge
+      e = icc::launch_merge_keys(seed_lists, pl.n_partitions, nq, k, partials + (size_t)pl.n_partitions * list_block,
+                                 static_cast<uint64_t*>(c->thr.p), c->stream);
+      if (e != cudaSuccess) return fail(IC_ERR_CUDA, "seed merge launch failed: %s", cudaGetErrorString(e));
+      c->launches += 1;
+      n_final_lists = pl.n_partitions + 1;
+    }
+    up.tile_begin = pl.seed_tiles;
+    up.tile_end = n_tiles;
+    up.thr_floor = pl.seed_tiles > 0 ? static_cast<const uint64_t*>(c->thr.p) : nullptr;
+    up.partials = partials;
     e = icc::launch_umma(up, c->stream);
     if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core scoring launch failed: %s", cudaGetErrorString(e));
     c->launches += 1;
   }
   profile_mark(c, c->ev_score, c->n_ev_score);
   profile_mark(c, c->ev_merge, c->n_ev_merge);
-  e = icc::launch_merge(partials, pl.n_partitions, nq, k, c->ids, out_ids, out_scores, c->stream);
+  e = icc::launch_merge(partials, n_final_lists, nq, k, c->ids, out_ids, out_scores, c->stream);
   if (e != cudaSuccess) return fail(IC_ERR_CUDA, "merge launch failed: %s", cudaGetErrorString(e));
   c->launches += 1;
   profile_mark(c, c->ev_merge, c->n_ev_merge);
@@ -479,6 +513,7 @@ void ic_cache_destroy(ic_cache_t* c) {
   release(c->q_bf16);
   release(c->q_f32);
   release(c->partials);
+  release(c->thr);
   release(c->stage_in);
   release(c->stage_ids);
   release(c->stage_scores);

@@ -40,8 +40,10 @@ struct UmmaParams {
   CUtensorMap tmap_q;     // [nq_pad, dim] bf16, box 64 x 128, 128-byte swizzle
   CUtensorMap tmap_slab;  // [capacity, dim] bf16, box 64 x 256, 128-byte swizzle
   int64_t n;
+  int64_t tile_begin, tile_end;   // 256-row tiles scored by this launch
   int dim;
   int q0, nq, k;          // queries [q0, q0 + n_query_tiles*128) of the staged batch
+  const uint64_t* thr_floor;      // optional [nq] keys: candidates at or below are discarded
   int n_query_tiles;
   int n_part;
   int n_stages;
@@ -56,6 +58,10 @@ cudaError_t umma_configure(int smem_optin);
 // Merge n_part partial lists per query into the final sorted top-k and gather ids.
 cudaError_t launch_merge(const uint64_t* partials, int n_part, int nq, int k, const int64_t* ids,
                          int64_t* out_ids, float* out_scores, cudaStream_t st);
+// Same merge, but the result stays in key form: out_keys [nq][k] (sorted, KEY_EMPTY padded)
+// and out_thr [nq] = the k-th key (KEY_EMPTY when fewer than k candidates exist).
+cudaError_t launch_merge_keys(const uint64_t* partials, int n_part, int nq, int k, uint64_t* out_keys,
+                              uint64_t* out_thr, cudaStream_t st);
 cudaError_t merge_configure(int smem_optin);
 
 }  // namespace icc

@@ -14,12 +14,12 @@ constexpr int MERGE_THREADS = 256;
 __global__ void __launch_bounds__(MERGE_THREADS)
 merge_topk_kernel(const uint64_t* __restrict__ partials, int n_part, int nq, int k,
                   const int64_t* __restrict__ ids, int64_t* __restrict__ out_ids,
-                  float* __restrict__ out_scores) {
+                  float* __restrict__ out_scores, uint64_t* __restrict__ out_keys,
+                  uint64_t* __restrict__ out_thr) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint64_t* cand = reinterpret_cast<uint64_t*>(smem_raw);                 // [n_part][k]
   uint32_t* pos = reinterpret_cast<uint32_t*>(cand + (size_t)n_part * k);  // [n_part]
-  __shared__ uint32_t win_slot[MAX_K];
-  __shared__ float win_score[MAX_K];
+  __shared__ uint64_t win_key[MAX_K];
 
   const int q = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
   const int total = n_part * k;
@@ -48,8 +48,7 @@ merge_topk_kernel(const uint64_t* __restrict__ partials, int n_part, int nq, int
       const uint32_t lo = (hi == top_hi) ? (uint32_t)best : 0u;
       const uint32_t top_lo = __reduce_max_sync(FULL_MASK, lo);
       if (hi == top_hi && lo == top_lo) {  // keys are unique, so exactly one lane wins
-        win_slot[r] = 0xffffffffu - top_lo;
-        win_score[r] = ord_to_score(top_hi);
+        win_key[r] = best;
         pos[best_p] += 1;
         best = KEY_EMPTY;
         best_p = -1;
@@ -60,16 +59,18 @@ merge_topk_kernel(const uint64_t* __restrict__ partials, int n_part, int nq, int
         }
       }
     }
-    for (int i = r + lane; i < k; i += 32) {  // fewer than k entries in the cache
-      win_slot[i] = 0xffffffffu;
-      win_score[i] = -INFINITY;
-    }
+    for (int i = r + lane; i < k; i += 32) win_key[i] = KEY_EMPTY;  // fewer than k candidates
   }
   __syncthreads();
+  if (out_keys) {  // intermediate merge: keep the key form
+    for (int i = tid; i < k; i += MERGE_THREADS) out_keys[(size_t)q * k + i] = win_key[i];
+    if (tid == 0) out_thr[q] = win_key[k - 1];
+    return;
+  }
   for (int i = tid; i < k; i += MERGE_THREADS) {
-    const uint32_t slot = win_slot[i];
-    out_scores[(size_t)q * k + i] = win_score[i];
-    out_ids[(size_t)q * k + i] = (slot == 0xffffffffu) ? (int64_t)-1 : ids[slot];
+    const uint64_t key = win_key[i];
+    out_scores[(size_t)q * k + i] = (key == KEY_EMPTY) ? -INFINITY : key_score(key);
+    out_ids[(size_t)q * k + i] = (key == KEY_EMPTY) ? (int64_t)-1 : ids[key_slot(key)];
   }
 }
 
@@ -86,7 +87,17 @@ cudaError_t launch_merge(const uint64_t* partials, int n_part, int nq, int k, co
                          int64_t* out_ids, float* out_scores, cudaStream_t st) {
   const size_t smem = (size_t)n_part * k * 8 + (size_t)n_part * 4;
   if (smem > (size_t)g_merge_smem_limit) return cudaErrorInvalidValue;
-  merge_topk_kernel<<<nq, MERGE_THREADS, smem, st>>>(partials, n_part, nq, k, ids, out_ids, out_scores);
+  merge_topk_kernel<<<nq, MERGE_THREADS, smem, st>>>(partials, n_part, nq, k, ids, out_ids, out_scores, nullptr,
+                                                     nullptr);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_merge_keys(const uint64_t* partials, int n_part, int nq, int k, uint64_t* out_keys,
+                              uint64_t* out_thr, cudaStream_t st) {
+  const size_t smem = (size_t)n_part * k * 8 + (size_t)n_part * 4;
+  if (smem > (size_t)g_merge_smem_limit || !out_keys || !out_thr) return cudaErrorInvalidValue;
+  merge_topk_kernel<<<nq, MERGE_THREADS, smem, st>>>(partials, n_part, nq, k, nullptr, nullptr, nullptr, out_keys,
+                                                     out_thr);
   return cudaGetLastError();
 }
 

@@ -43,7 +43,8 @@ struct UmmaSmemTail {
 
 __global__ void __launch_bounds__(UM_THREADS, 1)
 umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_slab,
-                       int64_t n, int dim, int nq, int k, int n_query_tiles, int n_part, int n_stages, int qcap,
+                       int64_t n, int64_t tile_begin, int64_t tile_end, int dim, int nq, int k, int n_query_tiles,
+                       int n_part, int n_stages, int qcap, const uint64_t* __restrict__ thr_floor_in,
                        uint64_t* __restrict__ partials, int* dev_status) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -56,7 +57,7 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int qt = blockIdx.x % n_query_tiles;     // query tile of this CTA
   const int part = blockIdx.x / n_query_tiles;   // row partition of this CTA
-  const int64_t n_tiles = (n + UM_RT - 1) / UM_RT;
+  // this launch scores row tiles [tile_begin, tile_end); CTA (part, qt) takes every n_part-th
   const int n_kc = (dim + UM_KC - 1) / UM_KC;
 
   if (tid == 0) {
@@ -88,7 +89,7 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     if (lane == 0) {
       int64_t it = 0;
       bool ok = true;
-      for (int64_t tile = part; tile < n_tiles && ok; tile += n_part) {
+      for (int64_t tile = tile_begin + part; tile < tile_end && ok; tile += n_part) {
         for (int kc = 0; kc < n_kc; ++kc, ++it) {
           const int s = (int)(it % n_stages);
           const uint32_t ph = (uint32_t)((it / n_stages) & 1);
@@ -119,7 +120,7 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       int64_t it = 0;
       int64_t lt = 0;
       bool ok = true;
-      for (int64_t tile = part; tile < n_tiles && ok; tile += n_part, ++lt) {
+      for (int64_t tile = tile_begin + part; tile < tile_end && ok; tile += n_part, ++lt) {
         const int buf = (int)(lt & 1);
         const uint32_t bph = (uint32_t)((lt >> 1) & 1);
         ok = mbar_wait(&tail->acc_empty[buf], bph ^ 1u, abort_flag);
@@ -169,8 +170,12 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     uint64_t* warp_lists = lists + (size_t)(warp * 32) * k;
     uint64_t* my_list = warp_lists + lane;                              // entry i at my_list[i * 32]
     uint64_t* my_queue = queues + (size_t)(warp * 32) * qcap + lane;    // entry i at my_queue[i * 32]
-    float thr_score = real ? -INFINITY : __int_as_float(0x7fc00000);   // NaN never admits
-    uint64_t thr_key = KEY_EMPTY;
+    // A seeding pass over a sample of the rows may have established that k entries with keys
+    // >= thr_floor exist: nothing at or below that key can be in the final top-k.
+    const uint64_t thr_floor = (real && thr_floor_in) ? thr_floor_in[q] : KEY_EMPTY;
+    uint64_t thr_key = thr_floor;
+    float thr_score = !real ? __int_as_float(0x7fc00000)               // NaN never admits
+                            : (thr_floor == KEY_EMPTY ? -INFINITY : key_score(thr_floor));
     int min_pos = 0;
     int cnt = 0;
     auto drain = [&]() {
@@ -185,16 +190,16 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             const uint64_t e = my_list[j * 32];
             if (e < m) { m = e; mp = j; }
           }
-          thr_key = m;
           min_pos = mp;
-          thr_score = (m == KEY_EMPTY) ? -INFINITY : key_score(m);
+          thr_key = m > thr_floor ? m : thr_floor;
+          thr_score = (thr_key == KEY_EMPTY) ? -INFINITY : key_score(thr_key);
         }
       }
       cnt = 0;
     };
     int64_t lt = 0;
     bool ok = true;
-    for (int64_t tile = part; tile < n_tiles; tile += n_part, ++lt) {
+    for (int64_t tile = tile_begin + part; tile < tile_end; tile += n_part, ++lt) {
       const int buf = (int)(lt & 1);
       const uint32_t bph = (uint32_t)((lt >> 1) & 1);
       ok = mbar_wait(&tail->acc_full[buf], bph, abort_flag);
@@ -279,8 +284,8 @@ cudaError_t launch_umma(const UmmaParams& p, cudaStream_t st) {
   const size_t need = 1024 + (size_t)p.n_stages * UM_STAGE_BYTES + (size_t)UM_QT * (p.k + p.queue_cap) * 8 + sizeof(UmmaSmemTail);
   if (need > (size_t)p.smem_bytes) return cudaErrorInvalidValue;
   umma_score_topk_kernel<<<p.n_part * p.n_query_tiles, UM_THREADS, p.smem_bytes, st>>>(
-      p.tmap_q, p.tmap_slab, p.n, p.dim, p.nq, p.k, p.n_query_tiles, p.n_part, p.n_stages, p.queue_cap, p.partials,
-      p.dev_status);
+      p.tmap_q, p.tmap_slab, p.n, p.tile_begin, p.tile_end, p.dim, p.nq, p.k, p.n_query_tiles, p.n_part, p.n_stages,
+      p.queue_cap, p.thr_floor, p.partials, p.dev_status);
   return cudaGetLastError();
 }
 

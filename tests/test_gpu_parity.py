@@ -85,6 +85,23 @@ def test_query_tiling(path, nq, k):
     run_and_check(x, q, k, path=PATHS[path], what=f"qtile/{path}/nq{nq}")
 
 
+@pytest.mark.parametrize("order", ["random", "best_first", "best_last"])
+@pytest.mark.parametrize("nq,k", [(8, 10), (130, 64)])
+def test_threshold_seeding_pass(order, nq, k):
+    # enough row tiles per CTA that the tensor-core path scores a sample first and starts the
+    # main pass from the sample's k-th best; with the best rows all inside (or all outside)
+    # the sample, the final merge must still return the exact top-k
+    from paper_2501_12689_b200 import ic_cache_plan
+    n, dim = 400_003, 64
+    assert ic_cache_plan(dim, n, nq, k, IC_PATH_UMMA)["seed_tiles"] > 0
+    x, q = _gauss(n, dim, nq, seed=55)
+    if order != "random":
+        s0 = (x.float() @ q[0].float())
+        idx = torch.argsort(s0, descending=(order == "best_first"))
+        x = x[idx].contiguous()
+    run_and_check(x, q, k, path=IC_PATH_UMMA, sample_queries=[0, 1, nq // 2, nq - 1], what=f"seed/{order}/nq{nq}")
+
+
 def test_more_queries_than_one_window():
     x, q = _gauss(3_001, 64, 1030, seed=60)
     run_and_check(x, q, 4, path=IC_PATH_UMMA, sample_queries=[0, 1, 127, 128, 1023, 1024, 1029], what="window")
