@@ -176,26 +176,41 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     uint64_t thr_key = thr_floor;
     float thr_score = !real ? __int_as_float(0x7fc00000)               // NaN never admits
                             : (thr_floor == KEY_EMPTY ? -INFINITY : key_score(thr_floor));
-    int min_pos = 0;
     int cnt = 0;
+    // The list is a binary min-heap (root = entry 0 = smallest kept key): admitting a candidate
+    // replaces the root and sifts it down, O(log k) shared-memory steps.  An all-empty list is
+    // a valid heap, so no separate fill phase exists.
     auto drain = [&]() {
       for (int i = 0; i < cnt; ++i) {
         const uint64_t key = my_queue[i * 32];
         if (key > thr_key) {
-          my_list[min_pos * 32] = key;
-          uint64_t m = ~0ull;
-          int mp = 0;
-#pragma unroll 4
-          for (int j = 0; j < k; ++j) {
-            const uint64_t e = my_list[j * 32];
-            if (e < m) { m = e; mp = j; }
+          int pos = 0;
+          uint64_t root = key;
+          while (true) {
+            const int l = 2 * pos + 1;
+            if (l >= k) break;
+            const uint64_t cl = my_list[l * 32];
+            const uint64_t cr = (l + 1 < k) ? my_list[(l + 1) * 32] : ~0ull;
+            const bool right = cr < cl;
+            const uint64_t cv = right ? cr : cl;
+            if (cv >= key) break;
+            my_list[pos * 32] = cv;
+            if (pos == 0) root = cv;
+            pos = right ? l + 1 : l;
           }
-          min_pos = mp;
-          thr_key = m > thr_floor ? m : thr_floor;
+          my_list[pos * 32] = key;
+          thr_key = root > thr_floor ? root : thr_floor;
           thr_score = (thr_key == KEY_EMPTY) ? -INFINITY : key_score(thr_key);
         }
       }
       cnt = 0;
+    };
+    auto consider = [&](float s, int64_t col) {
+      if (s >= thr_score) {
+        if (cnt == qcap) drain();
+        my_queue[cnt * 32] = make_key(s, (uint32_t)col);
+        ++cnt;
+      }
     };
     int64_t lt = 0;
     bool ok = true;
@@ -226,17 +241,19 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           for (int c = 0; c < 32; ++c)
             if (col0 + c >= n) v[c] = 0x7fc00000u;
         }
-        float best = __uint_as_float(v[0]);
+        // maxima of the eight groups of four columns, then of the whole batch
+        float g[8];
 #pragma unroll
-        for (int c = 1; c < 32; ++c) best = fmaxf(best, __uint_as_float(v[c]));
+        for (int j = 0; j < 8; ++j)
+          g[j] = fmaxf(fmaxf(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1])),
+                       fmaxf(__uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
+        const float best = fmaxf(fmaxf(fmaxf(g[0], g[1]), fmaxf(g[2], g[3])), fmaxf(fmaxf(g[4], g[5]), fmaxf(g[6], g[7])));
         if (!__any_sync(FULL_MASK, best >= thr_score)) continue;   // common case: nothing passes
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          const float s = __uint_as_float(v[c]);
-          if (s >= thr_score) {
-            if (cnt == qcap) drain();
-            my_queue[cnt * 32] = make_key(s, (uint32_t)(col0 + c));
-            ++cnt;
+        for (int j = 0; j < 8; ++j) {
+          if (g[j] >= thr_score) {
+#pragma unroll
+            for (int c = 4 * j; c < 4 * j + 4; ++c) consider(__uint_as_float(v[c]), col0 + c);
           }
         }
         if (__any_sync(FULL_MASK, 2 * cnt >= qcap)) drain();
