@@ -205,13 +205,6 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       }
       cnt = 0;
     };
-    auto consider = [&](float s, int64_t col) {
-      if (s >= thr_score) {
-        if (cnt == qcap) drain();
-        my_queue[cnt * 32] = make_key(s, (uint32_t)col);
-        ++cnt;
-      }
-    };
     int64_t lt = 0;
     bool ok = true;
     for (int64_t tile = tile_begin + part; tile < tile_end; tile += n_part, ++lt) {
@@ -249,11 +242,24 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                        fmaxf(__uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
         const float best = fmaxf(fmaxf(fmaxf(g[0], g[1]), fmaxf(g[2], g[3])), fmaxf(fmaxf(g[4], g[5]), fmaxf(g[6], g[7])));
         if (!__any_sync(FULL_MASK, best >= thr_score)) continue;   // common case: nothing passes
+        // Control flow below is warp-uniform: a drain is always entered by all 32 lanes, each
+        // working through its own queue, so lanes never wait for one another's list updates.
+        // A group of four columns adds at most four entries; the queue is drained whenever
+        // some lane could not take another group (or, for queues shorter than four, another
+        // entry).
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-          if (g[j] >= thr_score) {
+          if (__any_sync(FULL_MASK, g[j] >= thr_score)) {
 #pragma unroll
-            for (int c = 4 * j; c < 4 * j + 4; ++c) consider(__uint_as_float(v[c]), col0 + c);
+            for (int c = 4 * j; c < 4 * j + 4; ++c) {
+              const float s = __uint_as_float(v[c]);
+              if (s >= thr_score) {
+                my_queue[cnt * 32] = make_key(s, (uint32_t)(col0 + c));
+                ++cnt;
+              }
+              if (qcap < 4 && __any_sync(FULL_MASK, cnt >= qcap)) drain();
+            }
+            if (qcap >= 4 && __any_sync(FULL_MASK, cnt + 4 > qcap)) drain();
           }
         }
         if (__any_sync(FULL_MASK, 2 * cnt >= qcap)) drain();
