@@ -133,6 +133,37 @@ int ic_cache_query(ic_cache_t* c, const void* q, int32_t nq, int32_t k, int64_t*
 int ic_cache_query_host(ic_cache_t* c, const void* q_host, int32_t nq, int32_t k,
                         int64_t* out_ids_host, float* out_scores_host);
 
+/*
+ * ic_cache_query without any allocation (the paper has no counterpart; this exists for
+ * deployment).  Some callers must not allocate device memory at query time: a serving
+ * process whose framework has already reserved the whole GPU for its own memory pool (so a
+ * late cudaMalloc fails), or a latency-critical loop whose rules forbid calls that may
+ * synchronise the device, which cudaMalloc and cudaFree do.  ic_cache_query grows the
+ * library's scratch buffers on the first call of a larger shape; this variant never does.
+ * Its scratch (query staging, partial top-k lists, seed thresholds) is carved out of one
+ * fixed array of IC_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that
+ * loads the library holds that much memory until the process exits, whether or not this
+ * call is ever used.
+ *
+ * Arguments, results and ordering are exactly those of ic_cache_query (device pointers).
+ * Differences:
+ *   - a query whose scratch need exceeds IC_STATIC_SCRATCH_BYTES returns IC_ERR_NOMEM and
+ *     enqueues nothing; nq above 1024 returns IC_ERR_INVALID.  The need is about
+ *     6*dim*nq bytes of query staging plus 8*k*nq bytes per partial list, with up to
+ *     2*(SM count / ceil(nq/128)) + 1 lists; 64 queries, k = 10, dim = 768 need about 2 MB.
+ *   - the first call on a device looks up the array's device address (once per device, with
+ *     that device current); make that first call outside any stream capture.
+ *   - every handle, stream and thread of the process shares the one array per GPU, and it
+ *     keeps the previous call's contents.  Each call writes every word before reading it, so
+ *     nothing needs clearing, but two calls whose kernels overlap on the GPU (different
+ *     streams or handles) race on the scratch and return garbage: keep them ordered.
+ *   - it calls no cudaMalloc, cudaFree, event creation or other allocating routine, and
+ *     ignores ic_cache_set_profiling.
+ */
+#define IC_STATIC_SCRATCH_BYTES (8u << 20)
+int ic_cache_query_static(ic_cache_t* c, const void* q, int32_t nq, int32_t k, int64_t* out_ids,
+                          float* out_scores);
+
 /* ic_cache_insert for HOST buffers; synchronises the stream before returning. */
 int ic_cache_insert_host(ic_cache_t* c, const void* emb_host, const int64_t* ids_host, int64_t n);
 

@@ -22,6 +22,7 @@ IC_ERR_CUDA, IC_ERR_UNSUPPORTED, IC_ERR_TIMEOUT = -4, -5, -6
 IC_BF16, IC_F32 = 0, 1
 IC_PATH_AUTO, IC_PATH_GENERIC, IC_PATH_SCAN, IC_PATH_UMMA = 0, 1, 2, 3
 IC_MAX_K, IC_MAX_DIM = 128, 4096
+IC_STATIC_SCRATCH_BYTES = 8 << 20
 PATH_NAMES = {IC_PATH_AUTO: "auto", IC_PATH_GENERIC: "generic", IC_PATH_SCAN: "scan", IC_PATH_UMMA: "umma"}
 
 
@@ -61,6 +62,8 @@ SIGNATURES = {
     "ic_cache_insert": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64]),
     "ic_cache_query": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
                                       ctypes.c_void_p, ctypes.c_void_p]),
+    "ic_cache_query_static": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
+                                             ctypes.c_void_p, ctypes.c_void_p]),
     "ic_cache_query_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
                                            ctypes.c_void_p, ctypes.c_void_p]),
     "ic_cache_insert_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64]),
@@ -143,6 +146,12 @@ def ic_cache_insert(h, emb: torch.Tensor, ids: torch.Tensor, n: Optional[int] = 
 
 def ic_cache_query(h, q: torch.Tensor, nq: int, k: int, out_ids: torch.Tensor, out_scores: torch.Tensor) -> None:
     _check(load_library().ic_cache_query(h, _ptr(q), nq, k, _ptr(out_ids), _ptr(out_scores)))
+
+
+def ic_cache_query_static(h, q: torch.Tensor, nq: int, k: int, out_ids: torch.Tensor, out_scores: torch.Tensor) -> None:
+    """ic_cache_query with all scratch in the library's fixed static array: for callers that
+    must not allocate device memory at query time.  The caller supplies every buffer."""
+    _check(load_library().ic_cache_query_static(h, _ptr(q), nq, k, _ptr(out_ids), _ptr(out_scores)))
 
 
 def ic_cache_query_host(h, q: torch.Tensor, nq: int, k: int, out_ids: torch.Tensor, out_scores: torch.Tensor) -> None:
@@ -229,6 +238,20 @@ class ICCache:
             out_scores = torch.empty(nq, k, dtype=torch.float32, device=self.device)
         ic_cache_query(self._h, q, nq, k, out_ids, out_scores)
         return out_ids, out_scores
+
+    def query_static(self, q: torch.Tensor, k: int, out_ids: torch.Tensor, out_scores: torch.Tensor) -> None:
+        """Allocation-free query: results go into the caller's preallocated device tensors and
+        the library's scratch comes from its fixed static array (shared by all handles on the
+        GPU; keep calls ordered).  Raises ICCacheError(IC_ERR_NOMEM) if the shape needs more
+        scratch than the array holds."""
+        self._check_rows(q, True, "q")
+        nq = q.shape[0]
+        if out_ids.shape != (nq, k) or out_ids.dtype != torch.int64 or not out_ids.is_cuda or not out_ids.is_contiguous():
+            raise ValueError("out_ids must be a contiguous int64 device tensor of shape [nq, k]")
+        if out_scores.shape != (nq, k) or out_scores.dtype != torch.float32 or not out_scores.is_cuda \
+                or not out_scores.is_contiguous():
+            raise ValueError("out_scores must be a contiguous float32 device tensor of shape [nq, k]")
+        ic_cache_query_static(self._h, q, nq, k, out_ids, out_scores)
 
     def query_host(self, q: torch.Tensor, k: int, out_ids: Optional[torch.Tensor] = None,
                    out_scores: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:

@@ -8,6 +8,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -335,6 +336,135 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
   return IC_OK;
 }
 
+// ------------------------------------------------------------------ allocation-free query
+// Scratch of ic_cache_query_static: one fixed array in the library image, per GPU.  In host
+// code the symbol below is only a handle for the runtime, not a device address; the address
+// is looked up once per device with cudaGetSymbolAddress and cached here.
+static __device__ __align__(256) unsigned char g_static_scratch[IC_STATIC_SCRATCH_BYTES];
+constexpr int STATIC_MAX_DEVICES = 64;
+unsigned char* g_static_scratch_addr[STATIC_MAX_DEVICES] = {};
+std::mutex g_static_scratch_mutex;
+
+// Device address of the static scratch on `dev`, which must be the current device.
+int static_scratch_address(int dev, unsigned char** out) {
+  if (dev < 0 || dev >= STATIC_MAX_DEVICES) return fail(IC_ERR_UNSUPPORTED, "static scratch: device %d out of range", dev);
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (!g_static_scratch_addr[dev]) {
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess || !p) {
+      cudaGetLastError();
+      return fail(IC_ERR_CUDA, "cudaGetSymbolAddress of the static scratch failed on device %d: %s", dev, cudaGetErrorString(e));
+    }
+    g_static_scratch_addr[dev] = static_cast<unsigned char*>(p);
+  }
+  *out = g_static_scratch_addr[dev];
+  return IC_OK;
+}
+
+// One query window with all scratch taken from the static array.  Mirrors do_query_window
+// but never grows a buffer, creates an event or allocates in any other way.
+int do_query_window_static(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids, float* out_scores) {
+  ic_cache_plan_t pl;
+  int rc = plan_impl(c->dim, c->size, nq, k, c->forced_path, c->sm_count, c->smem_optin, &pl);
+  if (rc != IC_OK) return rc;
+  const int nq_pad = (nq + QUERY_TILE - 1) / QUERY_TILE * QUERY_TILE;
+  const size_t list_block = (size_t)nq * k;
+  auto round_up = [](size_t v) { return (v + 1023) & ~(size_t)1023; };
+  const size_t off_qbf16 = 0;
+  const size_t off_qf32 = off_qbf16 + round_up((size_t)nq_pad * c->dim * 2);
+  const size_t off_part = off_qf32 + round_up((size_t)nq * c->dim * 4);
+  const size_t off_thr = off_part + round_up((size_t)(2 * pl.n_partitions + 1) * list_block * 8);
+  const size_t need = off_thr + round_up((size_t)nq * 8);
+  if (need > (size_t)IC_STATIC_SCRATCH_BYTES)
+    return fail(IC_ERR_NOMEM, "query needs %zu bytes of scratch but the static scratch holds %u; use ic_cache_query or a smaller nq/k",
+                need, (unsigned)IC_STATIC_SCRATCH_BYTES);
+  unsigned char* base = nullptr;
+  if ((rc = static_scratch_address(c->device, &base)) != IC_OK) return rc;
+  void* q_bf16 = base + off_qbf16;
+  float* q_f32 = reinterpret_cast<float*>(base + off_qf32);
+  uint64_t* partials = reinterpret_cast<uint64_t*>(base + off_part);
+  uint64_t* thr = reinterpret_cast<uint64_t*>(base + off_thr);
+
+  cudaError_t e = icc::launch_convert_rows(q, c->input_dtype == IC_F32, nq, c->dim, c->normalize, q_bf16, q_f32, nq_pad,
+                                           c->stream);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "query preparation launch failed: %s", cudaGetErrorString(e));
+  c->launches += 1;
+  int n_final_lists = pl.n_partitions;
+  if (pl.path == IC_PATH_GENERIC) {
+    for (int q0 = 0; q0 < nq; q0 += GENERIC_QB) {
+      e = icc::launch_generic(c->slab, c->size, c->dim, q_f32, q0, nq, k, partials, pl.n_partitions, pl.smem_bytes,
+                              c->d_status, c->stream);
+      if (e != cudaSuccess) return fail(IC_ERR_CUDA, "generic scoring launch failed: %s", cudaGetErrorString(e));
+      c->launches += 1;
+    }
+  } else if (pl.path == IC_PATH_SCAN) {
+    for (int q0 = 0; q0 < nq; q0 += pl.query_tile) {
+      icc::ScanParams sp;
+      sp.slab = c->slab;
+      sp.n = c->size;
+      sp.dim = c->dim;
+      sp.q_f32 = q_f32;
+      sp.q0 = q0;
+      sp.nq = nq;
+      sp.qb = pl.query_tile;
+      sp.k = k;
+      sp.partials = partials;
+      sp.n_part = pl.n_partitions;
+      sp.n_stages = pl.n_stages;
+      sp.rows_per_stage = SCAN_ROWS_PER_STAGE;
+      sp.smem_bytes = pl.smem_bytes;
+      sp.dev_status = c->d_status;
+      e = icc::launch_scan(sp, c->stream);
+      if (e != cudaSuccess) return fail(IC_ERR_CUDA, "scan launch failed: %s", cudaGetErrorString(e));
+      c->launches += 1;
+    }
+  } else {
+    if (!c->have_tmap_slab) return fail(IC_ERR_UNSUPPORTED, "tensor-core path unavailable: no tensor map for the slab");
+    icc::UmmaParams up;
+    if ((rc = encode_2d(c, &up.tmap_q, q_bf16, (uint64_t)nq_pad, QUERY_TILE)) != IC_OK) return rc;
+    up.tmap_slab = c->tmap_slab;
+    up.n = c->size;
+    up.dim = c->dim;
+    up.q0 = 0;
+    up.nq = nq;
+    up.k = k;
+    up.n_query_tiles = pl.n_query_tiles;
+    up.n_part = pl.n_partitions;
+    up.n_stages = pl.n_stages;
+    up.queue_cap = pl.queue_cap;
+    up.smem_bytes = pl.smem_bytes;
+    up.dev_status = c->d_status;
+    const int64_t n_tiles = (c->size + ROW_TILE - 1) / ROW_TILE;
+    if (pl.seed_tiles > 0) {
+      uint64_t* seed_lists = partials + (size_t)(pl.n_partitions + 1) * list_block;
+      up.tile_begin = 0;
+      up.tile_end = pl.seed_tiles;
+      up.thr_floor = nullptr;
+      up.partials = seed_lists;
+      e = icc::launch_umma(up, c->stream);
+      if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core seeding launch failed: %s", cudaGetErrorString(e));
+      c->launches += 1;
+      e = icc::launch_merge_keys(seed_lists, pl.n_partitions, nq, k, partials + (size_t)pl.n_partitions * list_block, thr,
+                                 c->stream);
+      if (e != cudaSuccess) return fail(IC_ERR_CUDA, "seed merge launch failed: %s", cudaGetErrorString(e));
+      c->launches += 1;
+      n_final_lists = pl.n_partitions + 1;
+    }
+    up.tile_begin = pl.seed_tiles;
+    up.tile_end = n_tiles;
+    up.thr_floor = pl.seed_tiles > 0 ? thr : nullptr;
+    up.partials = partials;
+    e = icc::launch_umma(up, c->stream);
+    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core scoring launch failed: %s", cudaGetErrorString(e));
+    c->launches += 1;
+  }
+  e = icc::launch_merge(partials, n_final_lists, nq, k, c->ids, out_ids, out_scores, c->stream);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "merge launch failed: %s", cudaGetErrorString(e));
+  c->launches += 1;
+  return IC_OK;
+}
+
 int check_query_args(ic_cache* c, const void* q, int32_t nq, int32_t k, const void* out_ids, const void* out_scores) {
   if (!c) return fail(IC_ERR_INVALID, "NULL handle");
   if (nq < 0) return fail(IC_ERR_INVALID, "nq %d < 0", nq);
@@ -597,6 +727,17 @@ int ic_cache_query(ic_cache_t* c, const void* q, int32_t nq, int32_t k, int64_t*
     if (rc != IC_OK) return rc;
   }
   return IC_OK;
+}
+
+int ic_cache_query_static(ic_cache_t* c, const void* q, int32_t nq, int32_t k, int64_t* out_ids, float* out_scores) {
+  int rc = check_query_args(c, q, nq, k, out_ids, out_scores);
+  if (rc != IC_OK || nq == 0) return rc;
+  if (nq > WINDOW_MAX_NQ) return fail(IC_ERR_INVALID, "ic_cache_query_static takes at most %d queries per call", WINDOW_MAX_NQ);
+  DeviceGuard guard(c->device);
+  if (!is_device_ptr(q, c->device) || !is_device_ptr(out_ids, c->device) || !is_device_ptr(out_scores, c->device))
+    return fail(IC_ERR_INVALID, "q, out_ids and out_scores must be device pointers on device %d", c->device);
+  if ((rc = check_timeout(c)) != IC_OK) return rc;
+  return do_query_window_static(c, q, nq, k, out_ids, out_scores);
 }
 
 int ic_cache_query_host(ic_cache_t* c, const void* q_host, int32_t nq, int32_t k, int64_t* out_ids_host,
