@@ -96,6 +96,46 @@ __device__ __forceinline__ void locked_insert(uint64_t* list, int k, int* lock, 
   if (lane == 0) atomicExch(lock, 0);
 }
 
+// Tournament over the heads of sorted lists (list p starts at cand[p * stride], k entries each),
+// run by one warp; the winners go to win_key in order.  Lane l owns lists l, l+32,
+// ...; the current head of each owned list is kept in a register, so a round costs a few
+// compares, two warp max-reductions (score word, then slot word) and, for the winning lane
+// only, one shared-memory load of its list's next entry.  Returns the number of winners.
+template <int LPL>
+__device__ __forceinline__ int tournament_in_registers(const uint64_t* cand, int stride, int n_part, int k,
+                                                       int lane, uint64_t* win_key) {
+  uint64_t head[LPL];
+  int idx[LPL];
+#pragma unroll
+  for (int t = 0; t < LPL; ++t) {
+    const int p = lane + 32 * t;
+    head[t] = (p < n_part) ? cand[(size_t)p * stride] : KEY_EMPTY;
+    idx[t] = 0;
+  }
+  int r = 0;
+  for (; r < k; ++r) {
+    uint64_t best = head[0];
+#pragma unroll
+    for (int t = 1; t < LPL; ++t) best = head[t] > best ? head[t] : best;
+    const uint32_t hi = (uint32_t)(best >> 32);
+    const uint32_t top_hi = __reduce_max_sync(FULL_MASK, hi);
+    if (top_hi == 0) break;  // every list exhausted (warp-uniform)
+    const uint32_t lo = (hi == top_hi) ? (uint32_t)best : 0u;
+    const uint32_t top_lo = __reduce_max_sync(FULL_MASK, lo);
+    if (hi == top_hi && lo == top_lo) {  // keys are unique, so exactly one lane wins
+      win_key[r] = best;
+#pragma unroll
+      for (int t = 0; t < LPL; ++t) {
+        if (head[t] == best) {
+          idx[t] += 1;
+          head[t] = (idx[t] < k) ? cand[(size_t)(lane + 32 * t) * stride + idx[t]] : KEY_EMPTY;
+        }
+      }
+    }
+  }
+  return r;
+}
+
 // Unpack eight bf16 values held in a 16-byte vector into fp32.
 __device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float* x) {
   x[0] = __uint_as_float(v.x << 16);

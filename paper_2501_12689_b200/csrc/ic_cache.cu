@@ -35,6 +35,7 @@ constexpr int UMMA_STAGE_BYTES = (QUERY_TILE + ROW_TILE) * K_CHUNK * 2;  // 48 K
 constexpr int SCAN_MAX_Q = 4;
 constexpr int SCAN_MAX_DIM = 1024;
 constexpr int SCAN_ROWS_PER_STAGE = 32;
+constexpr int SCAN_CONSUMER_WARPS = 8;
 constexpr int GENERIC_QB = 4;
 constexpr int SEED_MIN_TILES_PER_CTA = 8;  // tcgen05 path: seed thresholds when a CTA has this many tiles
 constexpr int SEED_FRACTION = 16;          // share of the row tiles scored by the seeding pass
@@ -171,7 +172,7 @@ int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32
     out->n_partitions = std::max(1, std::min(sm_count, merge_lists_max));
     out->n_ctas = out->n_partitions;
     const int stage_bytes = SCAN_ROWS_PER_STAGE * dim * 2;
-    const int fixed = 2048 + SCAN_MAX_Q * k * 8;
+    const int fixed = 2048 + SCAN_CONSUMER_WARPS * SCAN_MAX_Q * k * 8;   // header + per-warp lists
     out->n_stages = std::min(8, (smem_optin - fixed) / stage_bytes);
     if (out->n_stages < 2) return fail(IC_ERR_UNSUPPORTED, "scan path: shared memory too small for dim %d", dim);
     out->smem_bytes = fixed + out->n_stages * stage_bytes;

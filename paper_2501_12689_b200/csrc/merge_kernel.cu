@@ -11,6 +11,37 @@ namespace icc {
 
 constexpr int MERGE_THREADS = 256;
 
+// Same tournament for any number of lists, with the list positions in shared memory.
+__device__ __forceinline__ int tournament_in_shared(const uint64_t* cand, uint32_t* pos, int n_part, int k, int lane,
+                                                    uint64_t* win_key) {
+  uint64_t best = KEY_EMPTY;
+  int best_p = -1;
+  for (int p = lane; p < n_part; p += 32) {
+    const uint64_t key = cand[(size_t)p * k];
+    if (key > best) { best = key; best_p = p; }
+  }
+  int r = 0;
+  for (; r < k; ++r) {
+    const uint32_t hi = (uint32_t)(best >> 32);
+    const uint32_t top_hi = __reduce_max_sync(FULL_MASK, hi);
+    if (top_hi == 0) break;
+    const uint32_t lo = (hi == top_hi) ? (uint32_t)best : 0u;
+    const uint32_t top_lo = __reduce_max_sync(FULL_MASK, lo);
+    if (hi == top_hi && lo == top_lo) {
+      win_key[r] = best;
+      pos[best_p] += 1;
+      best = KEY_EMPTY;
+      best_p = -1;
+      for (int p = lane; p < n_part; p += 32) {
+        const uint32_t j = pos[p];
+        const uint64_t key = (j < (uint32_t)k) ? cand[(size_t)p * k + j] : KEY_EMPTY;
+        if (key > best) { best = key; best_p = p; }
+      }
+    }
+  }
+  return r;
+}
+
 __global__ void __launch_bounds__(MERGE_THREADS)
 merge_topk_kernel(const uint64_t* __restrict__ partials, int n_part, int nq, int k,
                   const int64_t* __restrict__ ids, int64_t* __restrict__ out_ids,
@@ -34,31 +65,13 @@ merge_topk_kernel(const uint64_t* __restrict__ partials, int n_part, int nq, int
   __syncthreads();
 
   if (tid < 32) {
-    uint64_t best = KEY_EMPTY;
-    int best_p = -1;
-    for (int p = lane; p < n_part; p += 32) {
-      const uint64_t key = cand[(size_t)p * k];
-      if (key > best) { best = key; best_p = p; }
-    }
-    int r = 0;
-    for (; r < k; ++r) {
-      const uint32_t hi = (uint32_t)(best >> 32);
-      const uint32_t top_hi = __reduce_max_sync(FULL_MASK, hi);
-      if (top_hi == 0) break;  // every list exhausted (warp-uniform)
-      const uint32_t lo = (hi == top_hi) ? (uint32_t)best : 0u;
-      const uint32_t top_lo = __reduce_max_sync(FULL_MASK, lo);
-      if (hi == top_hi && lo == top_lo) {  // keys are unique, so exactly one lane wins
-        win_key[r] = best;
-        pos[best_p] += 1;
-        best = KEY_EMPTY;
-        best_p = -1;
-        for (int p = lane; p < n_part; p += 32) {
-          const uint32_t j = pos[p];
-          const uint64_t key = (j < (uint32_t)k) ? cand[(size_t)p * k + j] : KEY_EMPTY;
-          if (key > best) { best = key; best_p = p; }
-        }
-      }
-    }
+    int r;
+    if (n_part <= 32) r = tournament_in_registers<1>(cand, k, n_part, k, lane, win_key);
+    else if (n_part <= 64) r = tournament_in_registers<2>(cand, k, n_part, k, lane, win_key);
+    else if (n_part <= 96) r = tournament_in_registers<3>(cand, k, n_part, k, lane, win_key);
+    else if (n_part <= 128) r = tournament_in_registers<4>(cand, k, n_part, k, lane, win_key);
+    else if (n_part <= 160) r = tournament_in_registers<5>(cand, k, n_part, k, lane, win_key);
+    else r = tournament_in_shared(cand, pos, n_part, k, lane, win_key);
     for (int i = r + lane; i < k; i += 32) win_key[i] = KEY_EMPTY;  // fewer than k candidates
   }
   __syncthreads();

@@ -6,7 +6,8 @@
 // conflict-free 16-byte shared loads (lane l owns elements [8l, 8l+8) of every 256-element
 // span), multiply against queries held in registers as fp32, and reduce across the warp with
 // a transposing butterfly (one shuffle per (row, query) instead of five).  Candidates that
-// beat the CTA's current k-th best go into the CTA's sorted list for that query.
+// beat the warp's current k-th best go into the warp's own sorted list for that query (no
+// locks); when the scan ends, one warp per query merges the eight lists into the CTA's list.
 #include "common.cuh"
 #include "kernels.h"
 #include "pipeline.cuh"
@@ -24,7 +25,6 @@ constexpr int SCAN_MAX_QB = 4;
 struct ScanSmemHeader {
   uint64_t full[SCAN_MAX_STAGES];
   uint64_t empty[SCAN_MAX_STAGES];
-  int locks[SCAN_MAX_QB];
   int abort_flag;
 };
 
@@ -54,8 +54,8 @@ scan_score_topk_kernel(const __nv_bfloat16* __restrict__ slab, int64_t n, int di
                        uint64_t* __restrict__ partials, int n_stages, int* dev_status) {
   extern __shared__ __align__(128) unsigned char smem[];
   ScanSmemHeader* hdr = reinterpret_cast<ScanSmemHeader*>(smem);
-  uint64_t* lists = reinterpret_cast<uint64_t*>(smem + SCAN_LISTS_OFFSET);        // [SCAN_MAX_QB][k]
-  unsigned char* ring = smem + SCAN_LISTS_OFFSET + SCAN_MAX_QB * k * 8;
+  uint64_t* lists = reinterpret_cast<uint64_t*>(smem + SCAN_LISTS_OFFSET);        // [8 warps][SCAN_MAX_QB][k]
+  unsigned char* ring = smem + SCAN_LISTS_OFFSET + SCAN_CONSUMER_WARPS * SCAN_MAX_QB * k * 8;
   const int stage_bytes = SCAN_STAGE_ROWS * dim * 2;
   const int row_bytes = dim * 2;
   volatile int* abort_flag = &hdr->abort_flag;
@@ -69,8 +69,7 @@ scan_score_topk_kernel(const __nv_bfloat16* __restrict__ slab, int64_t n, int di
     hdr->abort_flag = 0;
     mbar_fence_init();
   }
-  if (tid < SCAN_MAX_QB) hdr->locks[tid] = 0;
-  for (int i = tid; i < SCAN_MAX_QB * k; i += SCAN_THREADS) lists[i] = KEY_EMPTY;
+  for (int i = tid; i < SCAN_CONSUMER_WARPS * SCAN_MAX_QB * k; i += SCAN_THREADS) lists[i] = KEY_EMPTY;
   __syncthreads();
 
   const int64_t n_pieces = (n + SCAN_STAGE_ROWS - 1) / SCAN_STAGE_ROWS;
@@ -127,7 +126,8 @@ scan_score_topk_kernel(const __nv_bfloat16* __restrict__ slab, int64_t n, int di
     const int my_row = my_val / QB;                // row within the warp's four
     const int my_q = my_val % QB;                  // query this lane reports for
     const bool reporter = (lane & ((1 << SHIFT) - 1)) == 0 && my_q < qcount;
-    uint64_t* my_list = lists + my_q * k;
+    uint64_t* warp_lists = lists + (size_t)warp * SCAN_MAX_QB * k;   // this warp's [SCAN_MAX_QB][k]
+    uint64_t thr = KEY_EMPTY;                                       // k-th best of list my_q
 
     int64_t it = 0;
     bool ok = true;
@@ -166,7 +166,6 @@ scan_score_topk_kernel(const __nv_bfloat16* __restrict__ slab, int64_t n, int di
       const float score = transpose_reduce<V>(acc, lane);
       const int64_t row = piece * SCAN_STAGE_ROWS + warp * SCAN_ROWS_PER_WARP + my_row;
       const uint64_t key = make_key(score, (uint32_t)row);
-      const uint64_t thr = *reinterpret_cast<volatile uint64_t*>(my_list + (k - 1));
       const bool hit = reporter && row < n && key > thr;
       unsigned hits = __ballot_sync(FULL_MASK, hit);
       while (hits) {
@@ -174,15 +173,18 @@ scan_score_topk_kernel(const __nv_bfloat16* __restrict__ slab, int64_t n, int di
         hits &= hits - 1;
         const uint64_t hkey = __shfl_sync(FULL_MASK, key, src);
         const int hq = __shfl_sync(FULL_MASK, my_q, src);
-        locked_insert(lists + hq * k, k, &hdr->locks[hq], hkey, lane, dev_status);
+        const uint64_t new_thr = warp_sorted_insert(warp_lists + hq * k, k, hkey, lane);
+        if (my_q == hq) thr = new_thr;
       }
     }
     if (!ok && lane == 0) report_status(dev_status, DEV_TIMEOUT_MBAR);
   }
   __syncthreads();
-  for (int i = tid; i < qcount * k; i += SCAN_THREADS) {
-    const int qq = i / k, j = i - qq * k;
-    partials[((size_t)blockIdx.x * nq + (q0 + qq)) * k + j] = lists[i];
+  // warp qq merges the eight warps' lists of query qq and writes the CTA's partial list
+  if (warp < qcount) {
+    uint64_t* dst = partials + ((size_t)blockIdx.x * nq + (q0 + warp)) * k;
+    const int won = tournament_in_registers<1>(lists + (size_t)warp * k, SCAN_MAX_QB * k, SCAN_CONSUMER_WARPS, k, lane, dst);
+    for (int i = won + lane; i < k; i += 32) dst[i] = KEY_EMPTY;
   }
 }
 
