@@ -172,7 +172,7 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     uint64_t* my_queue = queues + (size_t)(warp * 32) * qcap + lane;    // entry i at my_queue[i * 32]
     // A seeding pass over a sample of the rows may have established that k entries with keys
     // >= thr_floor exist: nothing at or below that key can be in the final top-k.
-    const uint64_t thr_floor = (real && thr_floor_in) ? thr_floor_in[q] : KEY_EMPTY;
+    uint64_t thr_floor = (real && thr_floor_in) ? thr_floor_in[q] : KEY_EMPTY;
     uint64_t thr_key = thr_floor;
     float thr_score = !real ? __int_as_float(0x7fc00000)               // NaN never admits
                             : (thr_floor == KEY_EMPTY ? -INFINITY : key_score(thr_floor));
@@ -180,25 +180,32 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     // The list is a binary min-heap (root = entry 0 = smallest kept key): admitting a candidate
     // replaces the root and sifts it down, O(log k) shared-memory steps.  An all-empty list is
     // a valid heap, so no separate fill phase exists.
+    // Place `key` at the root of the min-heap my_list[0 .. limit) and sift it down; returns the
+    // new root (the smallest entry).
+    auto sift_down = [&](uint64_t key, int limit) -> uint64_t {
+      int pos = 0;
+      uint64_t root = key;
+      while (true) {
+        const int l = 2 * pos + 1;
+        if (l >= limit) break;
+        const uint64_t cl = my_list[l * 32];
+        const uint64_t cr = (l + 1 < limit) ? my_list[(l + 1) * 32] : ~0ull;
+        const bool right = cr < cl;
+        const uint64_t cv = right ? cr : cl;
+        if (cv >= key) break;
+        my_list[pos * 32] = cv;
+        if (pos == 0) root = cv;
+        pos = right ? l + 1 : l;
+      }
+      my_list[pos * 32] = key;
+      return root;
+    };
     auto drain = [&]() {
       for (int i = 0; i < cnt; ++i) {
-        const uint64_t key = my_queue[i * 32];
+        const uint64_t raw = my_queue[i * 32];   // (score bits << 32) | slot
+        const uint64_t key = make_key(__uint_as_float((uint32_t)(raw >> 32)), (uint32_t)raw);
         if (key > thr_key) {
-          int pos = 0;
-          uint64_t root = key;
-          while (true) {
-            const int l = 2 * pos + 1;
-            if (l >= k) break;
-            const uint64_t cl = my_list[l * 32];
-            const uint64_t cr = (l + 1 < k) ? my_list[(l + 1) * 32] : ~0ull;
-            const bool right = cr < cl;
-            const uint64_t cv = right ? cr : cl;
-            if (cv >= key) break;
-            my_list[pos * 32] = cv;
-            if (pos == 0) root = cv;
-            pos = right ? l + 1 : l;
-          }
-          my_list[pos * 32] = key;
+          const uint64_t root = sift_down(key, k);
           thr_key = root > thr_floor ? root : thr_floor;
           thr_score = (thr_key == KEY_EMPTY) ? -INFINITY : key_score(thr_key);
         }
@@ -216,6 +223,56 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       tc_fence_after_sync();
       const uint32_t t_addr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * UM_RT);
       const int64_t row0 = tile * UM_RT;
+      if (lt == 0 && thr_floor_in == nullptr && k <= 16 && row0 + UM_RT <= n) {
+        // Cold start (empty lists, no seed threshold): read the tile once just to take the
+        // maximum of each group of 16 columns.  The k-th largest of the 16 group maxima is a
+        // safe floor - k different columns score at least that much - and only ~6 % of the
+        // columns pass it, instead of every column passing an empty list.
+        float m[16];
+#pragma unroll
+        for (int cb = 0; cb < UM_RT / 32; ++cb) {
+          uint32_t v[32];
+          tmem_ld_32x32(t_addr + (uint32_t)(cb * 32), v);
+          tmem_ld_wait();
+          float a = __uint_as_float(v[0]), b = __uint_as_float(v[16]);
+#pragma unroll
+          for (int c = 1; c < 16; ++c) {
+            a = fmaxf(a, __uint_as_float(v[c]));
+            b = fmaxf(b, __uint_as_float(v[16 + c]));
+          }
+          m[2 * cb] = a;
+          m[2 * cb + 1] = b;
+        }
+        // bitonic sorting network, descending, on registers
+#pragma unroll
+        for (int ls = 1; ls <= 4; ++ls) {
+#pragma unroll
+          for (int lj = 3; lj >= 0; --lj) {
+            if (lj < ls) {
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                const int j = i ^ (1 << lj);
+                if (j > i) {
+                  const bool desc = (i & (1 << ls)) == 0;
+                  const float hi = fmaxf(m[i], m[j]), lo = fminf(m[i], m[j]);
+                  m[i] = desc ? hi : lo;
+                  m[j] = desc ? lo : hi;
+                }
+              }
+            }
+          }
+        }
+        // m is sorted descending: its k-th entry is the largest of the entries k-1 .. 15
+        float tau = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) tau = fmaxf(tau, i >= k - 1 ? m[i] : -INFINITY);
+        if (real && tau == tau) {
+          // admit every key whose score is >= tau: the smallest such key has slot word 0
+          thr_floor = ((uint64_t)score_to_ord(tau) << 32) - 1;
+          thr_key = thr_floor;
+          thr_score = tau;
+        }
+      }
 #pragma unroll 1
       for (int cb = 0; cb < UM_RT / 32; ++cb) {
         uint32_t v[32];
@@ -228,54 +285,74 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           if (lane == 0) mbar_arrive(&tail->acc_empty[buf]);
         }
         const int64_t col0 = row0 + cb * 32;
-        if (col0 >= n) continue;                    // warp-uniform
-        if (n - col0 < 32) {                        // ragged last tile: columns past n never admit
+        const bool last_batch = cb == UM_RT / 32 - 1;
+        float g[8];                                   // maxima of the eight groups of four columns
+        bool active = col0 < n;                       // warp-uniform
+        if (active) {
+          if (n - col0 < 32) {                        // ragged last tile: columns past n never admit
 #pragma unroll
-          for (int c = 0; c < 32; ++c)
-            if (col0 + c >= n) v[c] = 0x7fc00000u;
-        }
-        // maxima of the eight groups of four columns, then of the whole batch
-        float g[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-          g[j] = fmaxf(fmaxf(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1])),
-                       fmaxf(__uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
-        const float best = fmaxf(fmaxf(fmaxf(g[0], g[1]), fmaxf(g[2], g[3])), fmaxf(fmaxf(g[4], g[5]), fmaxf(g[6], g[7])));
-        if (!__any_sync(FULL_MASK, best >= thr_score)) continue;   // common case: nothing passes
-        // Control flow below is warp-uniform: a drain is always entered by all 32 lanes, each
-        // working through its own queue, so lanes never wait for one another's list updates.
-        // A group of four columns adds at most four entries; the queue is drained whenever
-        // some lane could not take another group (or, for queues shorter than four, another
-        // entry).
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          if (__any_sync(FULL_MASK, g[j] >= thr_score)) {
-#pragma unroll
-            for (int c = 4 * j; c < 4 * j + 4; ++c) {
-              const float s = __uint_as_float(v[c]);
-              if (s >= thr_score) {
-                my_queue[cnt * 32] = make_key(s, (uint32_t)(col0 + c));
-                ++cnt;
-              }
-              if (qcap < 4 && __any_sync(FULL_MASK, cnt >= qcap)) drain();
-            }
-            if (qcap >= 4 && __any_sync(FULL_MASK, cnt + 4 > qcap)) drain();
+            for (int c = 0; c < 32; ++c)
+              if (col0 + c >= n) v[c] = 0x7fc00000u;
           }
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            g[j] = fmaxf(fmaxf(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1])),
+                         fmaxf(__uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
+          const float best = fmaxf(fmaxf(fmaxf(g[0], g[1]), fmaxf(g[2], g[3])), fmaxf(fmaxf(g[4], g[5]), fmaxf(g[6], g[7])));
+          active = __any_sync(FULL_MASK, best >= thr_score);   // common case: nothing passes
         }
-        if (__any_sync(FULL_MASK, 2 * cnt >= qcap)) drain();
+        // Everything below is warp-uniform control flow, and the queue is drained at one place
+        // only (the code stays small and a drain is always entered by all 32 lanes, each working
+        // through its own queue).  Columns are considered in order; whenever some lane's queue
+        // could not take another group of four (or, for queues shorter than four, another
+        // entry) the pass stops, the queues are drained and the pass resumes at c_next.
+        int c_next = 0;
+        while (true) {
+          bool need_drain = false;
+          if (active) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              if (!need_drain && 4 * j + 3 >= c_next && __any_sync(FULL_MASK, g[j] >= thr_score)) {
+#pragma unroll
+                for (int c = 4 * j; c < 4 * j + 4; ++c) {
+                  if (!need_drain && c >= c_next) {
+                    const float s = __uint_as_float(v[c]);
+                    if (s >= thr_score) {
+                      my_queue[cnt * 32] = ((uint64_t)v[c] << 32) | (uint32_t)(col0 + c);
+                      ++cnt;
+                    }
+                    if (qcap < 4 && __any_sync(FULL_MASK, cnt >= qcap)) {
+                      need_drain = true;
+                      c_next = c + 1;
+                    }
+                  }
+                }
+                if (!need_drain && qcap >= 4 && __any_sync(FULL_MASK, cnt + 4 > qcap)) {
+                  need_drain = true;
+                  c_next = 4 * j + 4;
+                }
+              }
+            }
+            if (!need_drain) {
+              active = false;
+              need_drain = __any_sync(FULL_MASK, 2 * cnt >= qcap);
+            }
+          }
+          // fresh thresholds for the next tile
+          if (!active && last_batch) need_drain = need_drain || __any_sync(FULL_MASK, cnt > 0);
+          if (need_drain) drain();
+          if (!active) break;
+        }
       }
-      drain();   // fresh thresholds for the next tile
     }
     if (!ok && lane == 0) report_status(dev_status, DEV_TIMEOUT_MBAR);
-    // sort each private list descending (insertion sort, lanes in parallel)
-    for (int i = 1; i < k; ++i) {
-      const uint64_t e = my_list[i * 32];
-      int j = i - 1;
-      while (j >= 0 && my_list[j * 32] < e) {
-        my_list[(j + 1) * 32] = my_list[j * 32];
-        --j;
-      }
-      my_list[(j + 1) * 32] = e;
+    // sort each private list descending, lanes in parallel: heapsort in place (the smallest
+    // entry goes to the end of the shrinking heap)
+    for (int end = k - 1; end > 0; --end) {
+      const uint64_t smallest = my_list[0];
+      const uint64_t moved = my_list[end * 32];
+      my_list[end * 32] = smallest;
+      sift_down(moved, end);
     }
     __syncwarp();
     // transpose out: the partial lists of this warp's queries are contiguous in global memory
