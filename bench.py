@@ -40,6 +40,7 @@ def parse_args():
     ap.add_argument("--workload", default="online")
     ap.add_argument("--nq", type=int, default=None, help="query batch size (default: largest of the workload's sweep)")
     ap.add_argument("--path", default="auto", choices=["auto", "generic", "scan", "umma"])
+    ap.add_argument("--rows", type=int, default=None, help="scale the workload's cache to this many rows (profiling aid)")
     ap.add_argument("--no-sweep", action="store_true", help="skip the secondary batch sizes")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -174,6 +175,8 @@ def run_ours(args):
     dist, rank, world, local = dist_setup(args.gpus)
     dev = torch.device("cuda", local)
     w = wl.WORKLOADS[args.workload]
+    if args.rows:
+        w = w.scaled(args.rows)
     nq = args.nq or max(w.q_sweep)
     steps = args.steps if args.steps is not None else 500
     warmup = max(args.warmup if args.warmup is not None else 10, 3)
@@ -369,6 +372,8 @@ def run_reference(args):
     from oracle.ic_oracle import default_threads
     from paper_2501_12689_b200 import workloads as wl
     w = wl.WORKLOADS[args.workload]
+    if args.rows:
+        w = w.scaled(args.rows)
     nq = args.nq or max(w.q_sweep)
     steps = args.steps if args.steps is not None else 8
     warmup = args.warmup if args.warmup is not None else 1
