@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -83,7 +84,8 @@ struct ic_cache {
   int* d_status = nullptr;
   int64_t launches = 0;
   EncodeTiledFn encode = nullptr;
-  CUtensorMap tmap_slab;
+  CUtensorMap tmap_slab;       // box of 256 rows
+  CUtensorMap tmap_slab_half;  // box of 128 rows, for CTA pairs
   bool have_tmap_slab = false;
   // optional per-kernel timing (ic_cache_set_profiling)
   bool profiling = false;
@@ -180,7 +182,14 @@ int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32
   } else {
     out->query_tile = QUERY_TILE;
     out->n_query_tiles = (window + QUERY_TILE - 1) / QUERY_TILE;
-    out->n_partitions = std::max(1, std::min(sm_count / out->n_query_tiles, merge_lists_max - 1));
+    // An even number of query tiles runs as CTA pairs (one 256-query MMA per pair): each CTA
+    // then stages only half of every row tile.
+    out->cta_group = (out->n_query_tiles % 2 == 0 && sm_count >= 2) ? 2 : 1;
+    if (const char* env = getenv("IC_CACHE_CTA_GROUP")) {   // tuning knob: "1" forces single CTAs
+      if (env[0] == '1' && env[1] == 0) out->cta_group = 1;
+    }
+    const int units = out->n_query_tiles / out->cta_group;                    // CTAs or pairs per partition
+    out->n_partitions = std::max(1, std::min((sm_count / out->cta_group) / units, merge_lists_max - 1));
     out->n_ctas = out->n_partitions * out->n_query_tiles;
     // Threshold seeding: with enough row tiles per CTA, first score 1/16 of them, merge that
     // sample's lists into its exact top-k and start the main pass from the sample's k-th key.
@@ -192,12 +201,13 @@ int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32
     // 1 KiB alignment slack + 256 B of barriers, the per-query lists, then as many candidate
     // queue entries per query (up to 8) as still leave room for two ring stages
     const int base = 1024 + 256 + QUERY_TILE * k * 8;
-    out->queue_cap = std::min(8, (smem_optin - base - 2 * UMMA_STAGE_BYTES) / (QUERY_TILE * 8));
+    const int stage_bytes = (QUERY_TILE + ROW_TILE / out->cta_group) * K_CHUNK * 2;   // 48 or 32 KiB
+    out->queue_cap = std::min(8, (smem_optin - base - 2 * stage_bytes) / (QUERY_TILE * 8));
     if (out->queue_cap < 1) return fail(IC_ERR_UNSUPPORTED, "tensor-core path: shared memory too small");
     const int fixed = base + QUERY_TILE * out->queue_cap * 8;
-    out->n_stages = std::min(6, (smem_optin - fixed) / UMMA_STAGE_BYTES);
+    out->n_stages = std::min(8, (smem_optin - fixed) / stage_bytes);
     if (out->n_stages < 2) return fail(IC_ERR_UNSUPPORTED, "tensor-core path: shared memory too small");
-    out->smem_bytes = fixed + out->n_stages * UMMA_STAGE_BYTES;
+    out->smem_bytes = fixed + out->n_stages * stage_bytes;
     out->n_launches = n_windows * (out->seed_tiles > 0 ? 2 : 1);
   }
   return IC_OK;
@@ -291,6 +301,8 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
     icc::UmmaParams up;
     if ((rc = encode_2d(c, &up.tmap_q, c->q_bf16.p, (uint64_t)nq_pad, QUERY_TILE)) != IC_OK) return rc;
     up.tmap_slab = c->tmap_slab;
+    up.tmap_slab_half = c->tmap_slab_half;
+    up.cta_group = pl.cta_group;
     up.n = c->size;
     up.dim = c->dim;
     up.q0 = 0;
@@ -425,6 +437,8 @@ int do_query_window_static(ic_cache* c, const void* q, int nq, int k, int64_t* o
     icc::UmmaParams up;
     if ((rc = encode_2d(c, &up.tmap_q, q_bf16, (uint64_t)nq_pad, QUERY_TILE)) != IC_OK) return rc;
     up.tmap_slab = c->tmap_slab;
+    up.tmap_slab_half = c->tmap_slab_half;
+    up.cta_group = pl.cta_group;
     up.n = c->size;
     up.dim = c->dim;
     up.q0 = 0;
@@ -611,7 +625,8 @@ ic_cache_t* ic_cache_create_ex(int32_t dim, int64_t capacity, const ic_cache_opt
       ok = false;
     } else {
       c->encode = reinterpret_cast<EncodeTiledFn>(fn);
-      ok = encode_2d(c, &c->tmap_slab, c->slab, (uint64_t)capacity, ROW_TILE) == IC_OK;
+      ok = encode_2d(c, &c->tmap_slab, c->slab, (uint64_t)capacity, ROW_TILE) == IC_OK &&
+           encode_2d(c, &c->tmap_slab_half, c->slab, (uint64_t)capacity, ROW_TILE / 2) == IC_OK;
       c->have_tmap_slab = ok;
     }
   }

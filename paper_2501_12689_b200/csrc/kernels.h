@@ -39,6 +39,8 @@ cudaError_t scan_configure(int smem_optin);
 struct UmmaParams {
   CUtensorMap tmap_q;     // [nq_pad, dim] bf16, box 64 x 128, 128-byte swizzle
   CUtensorMap tmap_slab;  // [capacity, dim] bf16, box 64 x 256, 128-byte swizzle
+  CUtensorMap tmap_slab_half;  // same tensor, box 64 x 128 (CTA pairs: each CTA loads half a tile)
+  int cta_group;          // 1, or 2 = CTA pairs sharing each row tile
   int64_t n;
   int64_t tile_begin, tile_end;   // 256-row tiles scored by this launch
   int dim;

@@ -14,6 +14,7 @@
 // Two 256-column accumulators alternate, so the epilogue of one row tile overlaps the MMAs
 // of the next.  CTA (p, t) scores query tile t against row tiles p, p + P, p + 2P, ...
 #include <math.h>
+#include <string.h>
 
 #include "common.cuh"
 #include "kernels.h"
@@ -28,7 +29,11 @@ constexpr int UM_KC = 64;             // elements per K chunk (128 bytes)
 constexpr int UM_A_BYTES = UM_QT * UM_KC * 2;   // 16 KiB
 constexpr int UM_B_BYTES = UM_RT * UM_KC * 2;   // 32 KiB
 constexpr int UM_STAGE_BYTES = UM_A_BYTES + UM_B_BYTES;
-constexpr int UM_MAX_STAGES = 6;
+// With CTA pairs (CG = 2) the MMA is 256 x 256: each CTA of the pair stages its own 128 queries
+// and only half of the 256 cache rows, so a stage is 32 KiB and each slab byte enters the pair
+// once for 256 queries.
+template <int CG> __host__ __device__ constexpr int um_stage_bytes() { return UM_A_BYTES + UM_B_BYTES / CG; }
+constexpr int UM_MAX_STAGES = 8;
 constexpr int UM_TMEM_COLS = 512;
 
 struct UmmaSmemTail {
@@ -41,6 +46,7 @@ struct UmmaSmemTail {
   int abort_flag;
 };
 
+template <int CG>
 __global__ void __launch_bounds__(UM_THREADS, 1)
 umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_slab,
                        int64_t n, int64_t tile_begin, int64_t tile_end, int dim, int nq, int k, int n_query_tiles,
@@ -48,26 +54,33 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                        uint64_t* __restrict__ partials, int* dev_status) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  unsigned char* ring = smem;                                                        // n_stages * 48 KiB
-  uint64_t* lists = reinterpret_cast<uint64_t*>(ring + (size_t)n_stages * UM_STAGE_BYTES);  // [128][k]
+  constexpr int STAGE_BYTES = um_stage_bytes<CG>();
+  unsigned char* ring = smem;                                                        // n_stages * STAGE_BYTES
+  uint64_t* lists = reinterpret_cast<uint64_t*>(ring + (size_t)n_stages * STAGE_BYTES);  // [128][k]
   uint64_t* queues = lists + (size_t)UM_QT * k;                                      // [128][qcap]
   UmmaSmemTail* tail = reinterpret_cast<UmmaSmemTail*>(queues + (size_t)UM_QT * qcap);
   volatile int* abort_flag = &tail->abort_flag;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int qt = blockIdx.x % n_query_tiles;     // query tile of this CTA
-  const int part = blockIdx.x / n_query_tiles;   // row partition of this CTA
+  // CG == 1: CTA b scores query tile b % nqt against partition b / nqt.  CG == 2: CTAs 2c and
+  // 2c+1 form a pair that scores query tiles 2*(c % (nqt/2)) + rank against partition
+  // c / (nqt/2); rank 0 issues the MMAs for both.
+  const uint32_t rank = (CG == 2) ? cluster_ctarank() : 0u;
+  const int unit = (CG == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int units_per_part = n_query_tiles / CG;
+  const int qt = (unit % units_per_part) * CG + (int)rank;   // query tile of this CTA
+  const int part = unit / units_per_part;                    // row partition of this CTA
   // this launch scores row tiles [tile_begin, tile_end); CTA (part, qt) takes every n_part-th
   const int n_kc = (dim + UM_KC - 1) / UM_KC;
 
   if (tid == 0) {
     for (int s = 0; s < n_stages; ++s) {
-      mbar_init(&tail->full[s], 1);
+      mbar_init(&tail->full[s], CG);       // one arrive.expect_tx per producing CTA
       mbar_init(&tail->empty[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&tail->acc_full[b], 1);
-      mbar_init(&tail->acc_empty[b], 4);
+      mbar_init(&tail->acc_empty[b], 4 * CG);  // one arrival per epilogue warp of every CTA
     }
     mbar_init(&tail->drain, 1);
     tail->abort_flag = 0;
@@ -78,10 +91,17 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     prefetch_tmap(&tmap_q);
     prefetch_tmap(&tmap_slab);
   }
-  if (warp == 5) tmem_alloc(&tail->tmem_base, UM_TMEM_COLS);
+  if (warp == 5) {
+    if (CG == 2) tmem_alloc_pair(&tail->tmem_base, UM_TMEM_COLS);
+    else tmem_alloc(&tail->tmem_base, UM_TMEM_COLS);
+  }
   tc_fence_before_sync();
   __syncthreads();
+  if (CG == 2) cluster_sync_all();   // the peer's barriers are initialised before anyone signals them
   tc_fence_after_sync();
+  // barriers the pair shares live in the rank-0 CTA
+  const uint32_t lead_full0 = (CG == 2) ? mapa_shared(smem_u32(&tail->full[0]), 0) : smem_u32(&tail->full[0]);
+  const uint32_t lead_acc_empty0 = (CG == 2) ? mapa_shared(smem_u32(&tail->acc_empty[0]), 0) : smem_u32(&tail->acc_empty[0]);
   const uint32_t tmem_base = tail->tmem_base;
 
   if (warp == 4) {
@@ -95,16 +115,23 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           const uint32_t ph = (uint32_t)((it / n_stages) & 1);
           ok = mbar_wait(&tail->empty[s], ph ^ 1u, abort_flag);
           if (!ok) break;
-          unsigned char* a_dst = ring + (size_t)s * UM_STAGE_BYTES;
-          mbar_arrive_expect_tx(&tail->full[s], UM_STAGE_BYTES);
-          tma_load_2d(a_dst, &tmap_q, kc * UM_KC, qt * UM_QT, &tail->full[s]);
-          tma_load_2d(a_dst + UM_A_BYTES, &tmap_slab, kc * UM_KC, (int)(tile * UM_RT), &tail->full[s]);
+          unsigned char* a_dst = ring + (size_t)s * STAGE_BYTES;
+          if (CG == 2) {
+            const uint32_t full = lead_full0 + (uint32_t)(s * 8);
+            mbar_arrive_expect_tx_cluster(full, STAGE_BYTES);
+            tma_load_2d_pair(a_dst, &tmap_q, kc * UM_KC, qt * UM_QT, full);
+            tma_load_2d_pair(a_dst + UM_A_BYTES, &tmap_slab, kc * UM_KC, (int)(tile * UM_RT) + (int)rank * (UM_RT / 2), full);
+          } else {
+            mbar_arrive_expect_tx(&tail->full[s], STAGE_BYTES);
+            tma_load_2d(a_dst, &tmap_q, kc * UM_KC, qt * UM_QT, &tail->full[s]);
+            tma_load_2d(a_dst + UM_A_BYTES, &tmap_slab, kc * UM_KC, (int)(tile * UM_RT), &tail->full[s]);
+          }
         }
       }
       if (!ok) {
         report_status(dev_status, DEV_TIMEOUT_MBAR);
         // loads already issued still write this CTA's shared memory: wait for them (bounded)
-        for (int64_t j = (it > n_stages ? it - n_stages : 0); j < it; ++j) {
+        for (int64_t j = (it > n_stages ? it - n_stages : 0); j < it && rank == 0; ++j) {
           const int s = (int)(j % n_stages);
           const long long t0 = clock64();
           while (!mbar_try_wait(&tail->full[s], (uint32_t)((j / n_stages) & 1)) &&
@@ -115,8 +142,8 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     }
   } else if (warp == 5) {
     // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16_f32(UM_QT, UM_RT);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16_f32(UM_QT * CG, UM_RT);
       int64_t it = 0;
       int64_t lt = 0;
       bool ok = true;
@@ -133,20 +160,27 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           ok = mbar_wait(&tail->full[s], ph, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          const uint32_t a_addr = smem_u32(ring + (size_t)s * UM_STAGE_BYTES);
+          const uint32_t a_addr = smem_u32(ring + (size_t)s * STAGE_BYTES);
           const uint64_t da = umma_desc_k_major_sw128(a_addr);
           const uint64_t db = umma_desc_k_major_sw128(a_addr + UM_A_BYTES);
 #pragma unroll
           for (int kk = 0; kk < UM_KC / 16; ++kk) {
             // 16 bf16 = 32 bytes further along K inside the swizzled 128-byte row
-            umma_bf16(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (kc | kk) != 0 ? 1u : 0u);
+            if (CG == 2) umma_bf16_pair(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (kc | kk) != 0 ? 1u : 0u);
+            else umma_bf16(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (kc | kk) != 0 ? 1u : 0u);
           }
-          umma_commit(&tail->empty[s]);   // stage reusable once these MMAs have read it
+          // stage reusable (in both CTAs of a pair) once these MMAs have read it
+          if (CG == 2) umma_commit_pair_both(&tail->empty[s]);
+          else umma_commit(&tail->empty[s]);
         }
-        if (ok) umma_commit(&tail->acc_full[buf]);
+        if (ok) {
+          if (CG == 2) umma_commit_pair_both(&tail->acc_full[buf]);
+          else umma_commit(&tail->acc_full[buf]);
+        }
       }
       // make sure nothing issued is still running before tensor memory is released
-      umma_commit(&tail->drain);
+      if (CG == 2) umma_commit_pair(&tail->drain);
+      else umma_commit(&tail->drain);
       {
         const long long t0 = clock64();
         while (!mbar_try_wait(&tail->drain, 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {
@@ -177,25 +211,30 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     float thr_score = !real ? __int_as_float(0x7fc00000)               // NaN never admits
                             : (thr_floor == KEY_EMPTY ? -INFINITY : key_score(thr_floor));
     int cnt = 0;
-    // The list is a binary min-heap (root = entry 0 = smallest kept key): admitting a candidate
-    // replaces the root and sifts it down, O(log k) shared-memory steps.  An all-empty list is
-    // a valid heap, so no separate fill phase exists.
-    // Place `key` at the root of the min-heap my_list[0 .. limit) and sift it down; returns the
-    // new root (the smallest entry).
+    // The list is a min-heap (root = entry 0 = smallest kept key): admitting a candidate replaces
+    // the root and sifts it down.  An all-empty list is a valid heap, so no fill phase exists.
+    // Place `key` at the root of the 4-ary min-heap my_list[0 .. limit) (children of entry i are
+    // 4i+1 .. 4i+4) and sift it down; returns the new root, the smallest entry.  Four children
+    // per level keep the chain of dependent shared-memory round trips short: log4(k) levels.
     auto sift_down = [&](uint64_t key, int limit) -> uint64_t {
       int pos = 0;
       uint64_t root = key;
       while (true) {
-        const int l = 2 * pos + 1;
-        if (l >= limit) break;
-        const uint64_t cl = my_list[l * 32];
-        const uint64_t cr = (l + 1 < limit) ? my_list[(l + 1) * 32] : ~0ull;
-        const bool right = cr < cl;
-        const uint64_t cv = right ? cr : cl;
+        const int c0 = 4 * pos + 1;
+        if (c0 >= limit) break;
+        const uint64_t v0 = my_list[c0 * 32];
+        const uint64_t v1 = (c0 + 1 < limit) ? my_list[(c0 + 1) * 32] : ~0ull;
+        const uint64_t v2 = (c0 + 2 < limit) ? my_list[(c0 + 2) * 32] : ~0ull;
+        const uint64_t v3 = (c0 + 3 < limit) ? my_list[(c0 + 3) * 32] : ~0ull;
+        const bool b01 = v1 < v0, b23 = v3 < v2;
+        const uint64_t m01 = b01 ? v1 : v0, m23 = b23 ? v3 : v2;
+        const int i01 = b01 ? c0 + 1 : c0, i23 = b23 ? c0 + 3 : c0 + 2;
+        const bool hi = m23 < m01;
+        const uint64_t cv = hi ? m23 : m01;
         if (cv >= key) break;
         my_list[pos * 32] = cv;
         if (pos == 0) root = cv;
-        pos = right ? l + 1 : l;
+        pos = hi ? i23 : i01;
       }
       my_list[pos * 32] = key;
       return root;
@@ -282,7 +321,7 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           // the accumulator has been read completely: hand it back to the MMA issuer
           tc_fence_before_sync();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&tail->acc_empty[buf]);
+          if (lane == 0) mbar_arrive_cluster(lead_acc_empty0 + (uint32_t)(buf * 8));
         }
         const int64_t col0 = row0 + cb * 32;
         const bool last_batch = cb == UM_RT / 32 - 1;
@@ -368,25 +407,49 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   }
   tc_fence_before_sync();
   __syncthreads();
+  if (CG == 2) cluster_sync_all();   // neither CTA leaves while the other may still signal it
   if (warp == 5) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, UM_TMEM_COLS);
+    if (CG == 2) tmem_dealloc_pair(tmem_base, UM_TMEM_COLS);
+    else tmem_dealloc(tmem_base, UM_TMEM_COLS);
   }
 }
 
 cudaError_t umma_configure(int smem_optin) {
-  return cudaFuncSetAttribute(umma_score_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+  cudaError_t e = cudaFuncSetAttribute(umma_score_topk_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(umma_score_topk_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+  return e;
 }
 
 cudaError_t launch_umma(const UmmaParams& p, cudaStream_t st) {
-  if (p.n_stages < 2 || p.n_stages > UM_MAX_STAGES) return cudaErrorInvalidValue;
-  if (p.queue_cap < 1) return cudaErrorInvalidValue;
-  const size_t need = 1024 + (size_t)p.n_stages * UM_STAGE_BYTES + (size_t)UM_QT * (p.k + p.queue_cap) * 8 + sizeof(UmmaSmemTail);
+  if (p.n_stages < 2 || p.n_stages > UM_MAX_STAGES || p.queue_cap < 1) return cudaErrorInvalidValue;
+  if (p.cta_group != 1 && p.cta_group != 2) return cudaErrorInvalidValue;
+  if (p.cta_group == 2 && (p.n_query_tiles % 2) != 0) return cudaErrorInvalidValue;
+  const int stage_bytes = p.cta_group == 2 ? um_stage_bytes<2>() : um_stage_bytes<1>();
+  const size_t need = 1024 + (size_t)p.n_stages * stage_bytes + (size_t)UM_QT * (p.k + p.queue_cap) * 8 + sizeof(UmmaSmemTail);
   if (need > (size_t)p.smem_bytes) return cudaErrorInvalidValue;
-  umma_score_topk_kernel<<<p.n_part * p.n_query_tiles, UM_THREADS, p.smem_bytes, st>>>(
-      p.tmap_q, p.tmap_slab, p.n, p.tile_begin, p.tile_end, p.dim, p.nq, p.k, p.n_query_tiles, p.n_part, p.n_stages,
-      p.queue_cap, p.thr_floor, p.partials, p.dev_status);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3((unsigned)(p.n_part * p.n_query_tiles), 1, 1);
+  cfg.blockDim = dim3(UM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = (size_t)p.smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  if (p.cta_group == 2) {
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, umma_score_topk_kernel<2>, p.tmap_q, p.tmap_slab_half, p.n, p.tile_begin, p.tile_end,
+                              p.dim, p.nq, p.k, p.n_query_tiles, p.n_part, p.n_stages, p.queue_cap, p.thr_floor,
+                              p.partials, p.dev_status);
+  }
+  return cudaLaunchKernelEx(&cfg, umma_score_topk_kernel<1>, p.tmap_q, p.tmap_slab, p.n, p.tile_begin, p.tile_end, p.dim,
+                            p.nq, p.k, p.n_query_tiles, p.n_part, p.n_stages, p.queue_cap, p.thr_floor, p.partials,
+                            p.dev_status);
 }
 
 }  // namespace icc
