@@ -87,6 +87,8 @@ typedef struct ic_cache_plan {
   int32_t queue_cap;     /* tensor-core path: candidate queue entries per query (else 0)   */
   int32_t seed_tiles;    /* tensor-core path: 256-row tiles scored first to seed the
                             per-query thresholds of the main pass (0 = single pass)        */
+  int32_t seed0_tiles;   /* tensor-core path: tiles of a first, smaller seeding pass that
+                            seeds the seeding pass itself (0 = none)                       */
   int32_t cta_group;     /* tensor-core path: 2 = CTA pairs issue one 256-query MMA and
                             split each row tile between them, 1 = single CTAs (else 0)     */
 } ic_cache_plan_t;

@@ -40,6 +40,8 @@ constexpr int SCAN_CONSUMER_WARPS = 8;
 constexpr int GENERIC_QB = 4;
 constexpr int SEED_MIN_TILES_PER_CTA = 8;  // tcgen05 path: seed thresholds when a CTA has this many tiles
 constexpr int SEED_FRACTION = 16;          // share of the row tiles scored by the seeding pass
+constexpr int SEED_TWO_LEVEL_TILES_PER_CTA = 4;
+constexpr size_t PACE_BYTES = 16384;       // progress words of the tensor-core path: one per CTA, 2048 at most
 
 struct DeviceGuard {
   int prev = -1;
@@ -79,7 +81,9 @@ struct ic_cache {
   bool own_slab = false;
   int64_t* ids = nullptr;
   bool own_ids = false;
-  Buffer q_bf16, q_f32, partials, thr, stage_in, stage_ids, stage_scores;
+  Buffer q_bf16, q_f32, partials, thr, pace, stage_in, stage_ids, stage_scores;
+  unsigned pace_epoch = 0;
+  int l2_bytes = 0;
   int* h_status = nullptr;  // pinned, mapped; kernels write a code when a bounded wait expires
   int* d_status = nullptr;
   int64_t launches = 0;
@@ -197,6 +201,9 @@ int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32
     if (n_tiles >= (int64_t)SEED_MIN_TILES_PER_CTA * out->n_partitions) {
       const int64_t t = n_tiles / SEED_FRACTION / out->n_partitions * out->n_partitions;
       out->seed_tiles = (int32_t)std::max<int64_t>(out->n_partitions, t);
+      // with several tiles per CTA in that sample, seed the sample itself from one tile per CTA
+      if (out->seed_tiles >= SEED_TWO_LEVEL_TILES_PER_CTA * out->n_partitions)
+        out->seed0_tiles = std::max(out->n_partitions, out->seed_tiles / SEED_FRACTION / out->n_partitions * out->n_partitions);
     }
     // 1 KiB alignment slack + 256 B of barriers, the per-query lists, then as many candidate
     // queue entries per query (up to 8) as still leave room for two ring stages
@@ -208,7 +215,7 @@ int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32
     out->n_stages = std::min(8, (smem_optin - fixed) / stage_bytes);
     if (out->n_stages < 2) return fail(IC_ERR_UNSUPPORTED, "tensor-core path: shared memory too small");
     out->smem_bytes = fixed + out->n_stages * stage_bytes;
-    out->n_launches = n_windows * (out->seed_tiles > 0 ? 2 : 1);
+    out->n_launches = n_windows * (1 + (out->seed_tiles > 0 ? 1 : 0) + (out->seed0_tiles > 0 ? 1 : 0));
   }
   return IC_OK;
 }
@@ -247,6 +254,85 @@ int do_insert(ic_cache* c, const void* emb, const int64_t* ids, int64_t n) {
   return IC_OK;
 }
 
+// Tensor-core scoring of one window: up to two threshold-seeding passes over growing samples of
+// the row tiles, each followed by a merge of its lists (plus the previous sample's merged list)
+// into the sample's exact top-k, then the main pass over the remaining tiles starting from
+// the last sample's k-th key.  Lists are blocks of nq*k keys inside `partials`:
+//   blocks 0 .. P-1      main pass            block P          last merged sample list
+//   blocks P+1 .. 2P     lists of a seeding pass                block 2P+1   first sample's merged list
+// On return *n_final_lists tells the final merge how many leading blocks to read.
+int run_umma_passes(ic_cache* c, const ic_cache_plan_t& pl, const void* q_bf16, int nq, int nq_pad, int k,
+                    uint64_t* partials, uint64_t* thr, unsigned long long* pace, int* n_final_lists) {
+  if (!c->have_tmap_slab) return fail(IC_ERR_UNSUPPORTED, "tensor-core path unavailable: no tensor map for the slab");
+  const int P = pl.n_partitions;
+  const size_t list_block = (size_t)nq * k;
+  icc::UmmaParams up;
+  int rc = encode_2d(c, &up.tmap_q, q_bf16, (uint64_t)nq_pad, QUERY_TILE);
+  if (rc != IC_OK) return rc;
+  up.tmap_slab = c->tmap_slab;
+  up.tmap_slab_half = c->tmap_slab_half;
+  up.cta_group = pl.cta_group;
+  up.n = c->size;
+  up.dim = c->dim;
+  up.q0 = 0;
+  up.nq = nq;
+  up.k = k;
+  up.n_query_tiles = pl.n_query_tiles;
+  up.n_part = P;
+  up.n_stages = pl.n_stages;
+  up.queue_cap = pl.queue_cap;
+  up.smem_bytes = pl.smem_bytes;
+  up.dev_status = c->d_status;
+  // CTAs of one partition may run an eighth of the partition's share of L2 apart (measured: with
+  // 18 partitions of 393 KB tiles, 3 tiles keep DRAM reads at the slab size, 8 tiles do not)
+  up.pace = pace;
+  const int64_t tile_bytes = (int64_t)ROW_TILE * c->dim * 2;
+  up.pace_window = (int)std::max<int64_t>(2, std::min<int64_t>(16, (int64_t)c->l2_bytes / 8 / ((int64_t)P * tile_bytes)));
+  if (const char* env = getenv("IC_CACHE_PACE_WINDOW")) {   // tuning knob: tiles; 0 switches pacing off
+    const int w = atoi(env);
+    if (w <= 0) up.pace = nullptr;
+    else up.pace_window = w;
+  }
+  const int64_t n_tiles = (c->size + ROW_TILE - 1) / ROW_TILE;
+  const int64_t bounds[3] = {pl.seed0_tiles, pl.seed_tiles, n_tiles};   // ends of pass 0, pass 1, main
+  uint64_t* pass_lists = partials + (size_t)(P + 1) * list_block;
+  uint64_t* first_merged = partials + (size_t)(2 * P + 1) * list_block;
+  uint64_t* last_merged = partials + (size_t)P * list_block;
+  int64_t begin = 0;
+  bool have_thr = false;
+  *n_final_lists = P;
+  for (int level = 0; level < 2; ++level) {
+    const int64_t end = bounds[level];
+    if (end <= begin) continue;   // this seeding level is not used
+    up.tile_begin = begin;
+    up.tile_end = end;
+    up.thr_floor = have_thr ? thr : nullptr;
+    up.partials = pass_lists;
+    up.pace_epoch = ++c->pace_epoch;
+    cudaError_t e = icc::launch_umma(up, c->stream);
+    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core seeding launch failed: %s", cudaGetErrorString(e));
+    c->launches += 1;
+    const bool last_seed = (end == pl.seed_tiles);
+    // pass lists (P blocks) are followed by the first sample's merged list when there is one
+    e = icc::launch_merge_keys(pass_lists, have_thr ? P + 1 : P, nq, k, last_seed ? last_merged : first_merged, thr,
+                               c->stream);
+    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "seed merge launch failed: %s", cudaGetErrorString(e));
+    c->launches += 1;
+    have_thr = true;
+    begin = end;
+    *n_final_lists = P + 1;
+  }
+  up.tile_begin = begin;
+  up.tile_end = n_tiles;
+  up.thr_floor = have_thr ? thr : nullptr;
+  up.partials = partials;
+  up.pace_epoch = ++c->pace_epoch;
+  cudaError_t e = icc::launch_umma(up, c->stream);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core scoring launch failed: %s", cudaGetErrorString(e));
+  c->launches += 1;
+  return IC_OK;
+}
+
 // One window of at most WINDOW_MAX_NQ queries, all pointers on the device.
 int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids, float* out_scores) {
   ic_cache_plan_t pl;
@@ -255,9 +341,9 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
   const int nq_pad = (nq + QUERY_TILE - 1) / QUERY_TILE * QUERY_TILE;
   if ((rc = ensure(c, c->q_bf16, (size_t)nq_pad * c->dim * 2, "query staging (bf16)")) != IC_OK) return rc;
   if ((rc = ensure(c, c->q_f32, (size_t)nq * c->dim * 4, "query staging (fp32)")) != IC_OK) return rc;
-  // lists of the main pass, one merged list of the seeding pass, lists of the seeding pass
+  // lists of the main pass, two merged sample lists, lists of a seeding pass
   const size_t list_block = (size_t)nq * k;   // keys of one partition
-  if ((rc = ensure(c, c->partials, (size_t)(2 * pl.n_partitions + 1) * list_block * 8, "partial top-k lists")) != IC_OK) return rc;
+  if ((rc = ensure(c, c->partials, (size_t)(2 * pl.n_partitions + 2) * list_block * 8, "partial top-k lists")) != IC_OK) return rc;
   if ((rc = ensure(c, c->thr, (size_t)nq * 8, "seed thresholds")) != IC_OK) return rc;
 
   cudaError_t e = icc::launch_convert_rows(q, c->input_dtype == IC_F32, nq, c->dim, c->normalize, c->q_bf16.p,
@@ -297,48 +383,9 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
       c->launches += 1;
     }
   } else {
-    if (!c->have_tmap_slab) return fail(IC_ERR_UNSUPPORTED, "tensor-core path unavailable: no tensor map for the slab");
-    icc::UmmaParams up;
-    if ((rc = encode_2d(c, &up.tmap_q, c->q_bf16.p, (uint64_t)nq_pad, QUERY_TILE)) != IC_OK) return rc;
-    up.tmap_slab = c->tmap_slab;
-    up.tmap_slab_half = c->tmap_slab_half;
-    up.cta_group = pl.cta_group;
-    up.n = c->size;
-    up.dim = c->dim;
-    up.q0 = 0;
-    up.nq = nq;
-    up.k = k;
-    up.n_query_tiles = pl.n_query_tiles;
-    up.n_part = pl.n_partitions;
-    up.n_stages = pl.n_stages;
-    up.queue_cap = pl.queue_cap;
-    up.smem_bytes = pl.smem_bytes;
-    up.dev_status = c->d_status;
-    const int64_t n_tiles = (c->size + ROW_TILE - 1) / ROW_TILE;
-    if (pl.seed_tiles > 0) {
-      // seeding pass over the first seed_tiles row tiles -> lists behind the main pass's
-      uint64_t* seed_lists = partials + (size_t)(pl.n_partitions + 1) * list_block;
-      up.tile_begin = 0;
-      up.tile_end = pl.seed_tiles;
-      up.thr_floor = nullptr;
-      up.partials = seed_lists;
-      e = icc::launch_umma(up, c->stream);
-      if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core seeding launch failed: %s", cudaGetErrorString(e));
-      c->launches += 1;
-      // exact top-k of the sample, kept as list number n_partitions of the final merge
-      e = icc::launch_merge_keys(seed_lists, pl.n_partitions, nq, k, partials + (size_t)pl.n_partitions * list_block,
-                                 static_cast<uint64_t*>(c->thr.p), c->stream);
-      if (e != cudaSuccess) return fail(IC_ERR_CUDA, "seed merge launch failed: %s", cudaGetErrorString(e));
-      c->launches += 1;
-      n_final_lists = pl.n_partitions + 1;
-    }
-    up.tile_begin = pl.seed_tiles;
-    up.tile_end = n_tiles;
-    up.thr_floor = pl.seed_tiles > 0 ? static_cast<const uint64_t*>(c->thr.p) : nullptr;
-    up.partials = partials;
-    e = icc::launch_umma(up, c->stream);
-    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core scoring launch failed: %s", cudaGetErrorString(e));
-    c->launches += 1;
+    rc = run_umma_passes(c, pl, c->q_bf16.p, nq, nq_pad, k, partials, static_cast<uint64_t*>(c->thr.p),
+                         static_cast<unsigned long long*>(c->pace.p), &n_final_lists);
+    if (rc != IC_OK) return rc;
   }
   profile_mark(c, c->ev_score, c->n_ev_score);
   profile_mark(c, c->ev_merge, c->n_ev_merge);
@@ -387,8 +434,9 @@ int do_query_window_static(ic_cache* c, const void* q, int nq, int k, int64_t* o
   const size_t off_qbf16 = 0;
   const size_t off_qf32 = off_qbf16 + round_up((size_t)nq_pad * c->dim * 2);
   const size_t off_part = off_qf32 + round_up((size_t)nq * c->dim * 4);
-  const size_t off_thr = off_part + round_up((size_t)(2 * pl.n_partitions + 1) * list_block * 8);
-  const size_t need = off_thr + round_up((size_t)nq * 8);
+  const size_t off_thr = off_part + round_up((size_t)(2 * pl.n_partitions + 2) * list_block * 8);
+  const size_t off_pace = off_thr + round_up((size_t)nq * 8);
+  const size_t need = off_pace + PACE_BYTES;
   if (need > (size_t)IC_STATIC_SCRATCH_BYTES)
     return fail(IC_ERR_NOMEM, "query needs %zu bytes of scratch but the static scratch holds %u; use ic_cache_query or a smaller nq/k",
                 need, (unsigned)IC_STATIC_SCRATCH_BYTES);
@@ -398,6 +446,7 @@ int do_query_window_static(ic_cache* c, const void* q, int nq, int k, int64_t* o
   float* q_f32 = reinterpret_cast<float*>(base + off_qf32);
   uint64_t* partials = reinterpret_cast<uint64_t*>(base + off_part);
   uint64_t* thr = reinterpret_cast<uint64_t*>(base + off_thr);
+  unsigned long long* pace = reinterpret_cast<unsigned long long*>(base + off_pace);
 
   cudaError_t e = icc::launch_convert_rows(q, c->input_dtype == IC_F32, nq, c->dim, c->normalize, q_bf16, q_f32, nq_pad,
                                            c->stream);
@@ -433,46 +482,8 @@ int do_query_window_static(ic_cache* c, const void* q, int nq, int k, int64_t* o
       c->launches += 1;
     }
   } else {
-    if (!c->have_tmap_slab) return fail(IC_ERR_UNSUPPORTED, "tensor-core path unavailable: no tensor map for the slab");
-    icc::UmmaParams up;
-    if ((rc = encode_2d(c, &up.tmap_q, q_bf16, (uint64_t)nq_pad, QUERY_TILE)) != IC_OK) return rc;
-    up.tmap_slab = c->tmap_slab;
-    up.tmap_slab_half = c->tmap_slab_half;
-    up.cta_group = pl.cta_group;
-    up.n = c->size;
-    up.dim = c->dim;
-    up.q0 = 0;
-    up.nq = nq;
-    up.k = k;
-    up.n_query_tiles = pl.n_query_tiles;
-    up.n_part = pl.n_partitions;
-    up.n_stages = pl.n_stages;
-    up.queue_cap = pl.queue_cap;
-    up.smem_bytes = pl.smem_bytes;
-    up.dev_status = c->d_status;
-    const int64_t n_tiles = (c->size + ROW_TILE - 1) / ROW_TILE;
-    if (pl.seed_tiles > 0) {
-      uint64_t* seed_lists = partials + (size_t)(pl.n_partitions + 1) * list_block;
-      up.tile_begin = 0;
-      up.tile_end = pl.seed_tiles;
-      up.thr_floor = nullptr;
-      up.partials = seed_lists;
-      e = icc::launch_umma(up, c->stream);
-      if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core seeding launch failed: %s", cudaGetErrorString(e));
-      c->launches += 1;
-      e = icc::launch_merge_keys(seed_lists, pl.n_partitions, nq, k, partials + (size_t)pl.n_partitions * list_block, thr,
-                                 c->stream);
-      if (e != cudaSuccess) return fail(IC_ERR_CUDA, "seed merge launch failed: %s", cudaGetErrorString(e));
-      c->launches += 1;
-      n_final_lists = pl.n_partitions + 1;
-    }
-    up.tile_begin = pl.seed_tiles;
-    up.tile_end = n_tiles;
-    up.thr_floor = pl.seed_tiles > 0 ? thr : nullptr;
-    up.partials = partials;
-    e = icc::launch_umma(up, c->stream);
-    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core scoring launch failed: %s", cudaGetErrorString(e));
-    c->launches += 1;
+    rc = run_umma_passes(c, pl, q_bf16, nq, nq_pad, k, partials, thr, pace, &n_final_lists);
+    if (rc != IC_OK) return rc;
   }
   e = icc::launch_merge(partials, n_final_lists, nq, k, c->ids, out_ids, out_scores, c->stream);
   if (e != cudaSuccess) return fail(IC_ERR_CUDA, "merge launch failed: %s", cudaGetErrorString(e));
@@ -567,6 +578,7 @@ ic_cache_t* ic_cache_create_ex(int32_t dim, int64_t capacity, const ic_cache_opt
   c->stream = static_cast<cudaStream_t>(o.stream);
   c->sm_count = prop.multiProcessorCount;
   c->smem_optin = (int)prop.sharedMemPerBlockOptin;
+  c->l2_bytes = prop.l2CacheSize;
 
   bool ok = true;
   if (o.slab) {
@@ -616,6 +628,18 @@ ic_cache_t* ic_cache_create_ex(int32_t dim, int64_t capacity, const ic_cache_opt
     }
   }
   if (ok) {
+    e = cudaMalloc(&c->pace.p, PACE_BYTES);
+    if (e == cudaSuccess) e = cudaMemset(c->pace.p, 0, PACE_BYTES);
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      fail(IC_ERR_NOMEM, "cudaMalloc of the pacing words failed: %s", cudaGetErrorString(e));
+      c->pace.p = nullptr;
+      ok = false;
+    } else {
+      c->pace.bytes = PACE_BYTES;
+    }
+  }
+  if (ok) {
     cudaDriverEntryPointQueryResult qres;
     void* fn = nullptr;
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
@@ -660,6 +684,7 @@ void ic_cache_destroy(ic_cache_t* c) {
   release(c->q_f32);
   release(c->partials);
   release(c->thr);
+  release(c->pace);
   release(c->stage_in);
   release(c->stage_ids);
   release(c->stage_scores);

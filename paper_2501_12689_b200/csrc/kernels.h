@@ -52,6 +52,9 @@ struct UmmaParams {
   int queue_cap;          // per-query candidate queue entries in shared memory
   int smem_bytes;
   uint64_t* partials;     // [n_part][nq][k]
+  unsigned long long* pace;   // optional [n_part][units per partition] progress words (L2 pacing hint)
+  unsigned pace_epoch;        // distinguishes this launch's progress words from older ones
+  int pace_window;            // tiles a CTA may run ahead of its slowest sibling
   int* dev_status;
 };
 cudaError_t launch_umma(const UmmaParams& p, cudaStream_t st);

@@ -35,6 +35,7 @@ constexpr int UM_STAGE_BYTES = UM_A_BYTES + UM_B_BYTES;
 template <int CG> __host__ __device__ constexpr int um_stage_bytes() { return UM_A_BYTES + UM_B_BYTES / CG; }
 constexpr int UM_MAX_STAGES = 8;
 constexpr int UM_TMEM_COLS = 512;
+constexpr long long PACE_LIMIT_CYCLES = 100000;   // ~50 us: longest a CTA holds back for a slower sibling
 
 struct UmmaSmemTail {
   uint64_t full[UM_MAX_STAGES];
@@ -51,7 +52,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
 umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_slab,
                        int64_t n, int64_t tile_begin, int64_t tile_end, int dim, int nq, int k, int n_query_tiles,
                        int n_part, int n_stages, int qcap, const uint64_t* __restrict__ thr_floor_in,
-                       uint64_t* __restrict__ partials, int* dev_status) {
+                       uint64_t* __restrict__ partials, unsigned long long* pace, unsigned pace_epoch,
+                       int pace_window, int* dev_status) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   constexpr int STAGE_BYTES = um_stage_bytes<CG>();
@@ -109,12 +111,35 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     if (lane == 0) {
       int64_t it = 0;
       bool ok = true;
-      for (int64_t tile = tile_begin + part; tile < tile_end && ok; tile += n_part) {
+      // Pacing.  The CTAs (or pairs) that score different query tiles against the same
+      // partition read the same row tiles; the tile comes from HBM once only while they stay
+      // within an L2-sized window of each other.  Each publishes how many tiles it has started
+      // and one that runs more than pace_window tiles ahead of the slowest holds its loads
+      // for a bounded time.  This is a bandwidth hint only: when the bound runs out it goes on.
+      const bool paced = (pace != nullptr) && units_per_part > 1 && rank == 0;
+      volatile unsigned long long* pace_row = paced ? pace + (size_t)part * units_per_part : nullptr;
+      const int my_unit = unit % units_per_part;
+      uint32_t ordinal = 0;
+      for (int64_t tile = tile_begin + part; tile < tile_end && ok; tile += n_part, ++ordinal) {
+        if (paced) pace_row[my_unit] = ((unsigned long long)pace_epoch << 32) | ordinal;
         for (int kc = 0; kc < n_kc; ++kc, ++it) {
           const int s = (int)(it % n_stages);
           const uint32_t ph = (uint32_t)((it / n_stages) & 1);
           ok = mbar_wait(&tail->empty[s], ph ^ 1u, abort_flag);
           if (!ok) break;
+          if (paced && kc == 0) {
+            const long long t0 = clock64();
+            while (true) {
+              uint32_t slowest = ordinal;
+              for (int u = 0; u < units_per_part; ++u) {
+                const unsigned long long v = pace_row[u];
+                const uint32_t o = ((uint32_t)(v >> 32) == pace_epoch) ? (uint32_t)v : 0u;   // not started yet
+                slowest = o < slowest ? o : slowest;
+              }
+              if (ordinal - slowest <= (uint32_t)pace_window || clock64() - t0 > PACE_LIMIT_CYCLES) break;
+              __nanosleep(200);
+            }
+          }
           unsigned char* a_dst = ring + (size_t)s * STAGE_BYTES;
           if (CG == 2) {
             const uint32_t full = lead_full0 + (uint32_t)(s * 8);
@@ -445,11 +470,11 @@ cudaError_t launch_umma(const UmmaParams& p, cudaStream_t st) {
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, umma_score_topk_kernel<2>, p.tmap_q, p.tmap_slab_half, p.n, p.tile_begin, p.tile_end,
                               p.dim, p.nq, p.k, p.n_query_tiles, p.n_part, p.n_stages, p.queue_cap, p.thr_floor,
-                              p.partials, p.dev_status);
+                              p.partials, p.pace, p.pace_epoch, p.pace_window, p.dev_status);
   }
   return cudaLaunchKernelEx(&cfg, umma_score_topk_kernel<1>, p.tmap_q, p.tmap_slab, p.n, p.tile_begin, p.tile_end, p.dim,
                             p.nq, p.k, p.n_query_tiles, p.n_part, p.n_stages, p.queue_cap, p.thr_floor, p.partials,
-                            p.dev_status);
+                            p.pace, p.pace_epoch, p.pace_window, p.dev_status);
 }
 
 }  // namespace icc

@@ -51,12 +51,14 @@ def test_plan_paths_and_shapes():
     p = pkg.ic_cache_plan(1024, 4_000_000, 256, 32)
     assert p["n_query_tiles"] == 2 and p["n_partitions"] == 74 and p["n_ctas"] == 148
     p = pkg.ic_cache_plan(768, 16_000_000, 1024, 64)
-    assert p["n_query_tiles"] == 8 and p["n_partitions"] == 18 and p["n_ctas"] == 144 and p["n_launches"] == 2
+    assert p["n_query_tiles"] == 8 and p["n_partitions"] == 18 and p["n_ctas"] == 144 and p["n_launches"] == 3
+    assert p["cta_group"] == 2 and 0 < p["seed0_tiles"] < p["seed_tiles"] and p["seed0_tiles"] % 18 == 0
     assert p["smem_bytes"] <= 232448
     assert p["seed_tiles"] > 0 and p["seed_tiles"] % 18 == 0 and p["seed_tiles"] * 256 * 15 < 16_000_000
     assert pkg.ic_cache_plan(768, 70_001, 64, 10)["seed_tiles"] == 0      # too few tiles per CTA
     p = pkg.ic_cache_plan(768, 16_000_000, 3000, 64)
-    assert p["n_launches"] == 6
+    assert p["n_launches"] == 9
+    assert pkg.ic_cache_plan(768, 1_000_000, 300, 10)["cta_group"] == 1    # odd number of query tiles
     p = pkg.ic_cache_plan(2048, 1000, 2, 5)          # too wide for the scan path
     assert p["path"] == pkg.IC_PATH_UMMA
     p = pkg.ic_cache_plan(64, 1000, 6, 128, path=pkg.IC_PATH_GENERIC)
