@@ -4,6 +4,7 @@
 // correct device path and so the fast paths can be cross-checked against something simple.
 #include "common.cuh"
 #include "kernels.h"
+#include "pipeline.cuh"
 
 namespace icc {
 
@@ -19,6 +20,8 @@ generic_score_topk_kernel(const __nv_bfloat16* __restrict__ slab, int64_t n, int
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int i = tid; i < GEN_QB * k; i += blockDim.x) lists[i] = KEY_EMPTY;
   if (tid < GEN_QB) locks[tid] = 0;
+  grid_dep_launch_dependents();
+  grid_dep_wait();
   __syncthreads();
 
   const int nchunk = dim >> 3;
@@ -71,9 +74,8 @@ generic_score_topk_kernel(const __nv_bfloat16* __restrict__ slab, int64_t n, int
 cudaError_t launch_generic(const void* slab, int64_t n, int dim, const float* q_f32, int q0, int nq,
                            int k, uint64_t* partials, int n_part, int smem_bytes, int* dev_status,
                            cudaStream_t st) {
-  generic_score_topk_kernel<<<n_part, GEN_WARPS * 32, smem_bytes, st>>>(
-      static_cast<const __nv_bfloat16*>(slab), n, dim, q_f32, q0, nq, k, partials, dev_status);
-  return cudaGetLastError();
+  return launch_overlapped(generic_score_topk_kernel, dim3(n_part), dim3(GEN_WARPS * 32), (size_t)smem_bytes, st, 1,
+                           static_cast<const __nv_bfloat16*>(slab), n, dim, q_f32, q0, nq, k, partials, dev_status);
 }
 
 }  // namespace icc

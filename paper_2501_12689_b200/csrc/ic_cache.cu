@@ -33,7 +33,8 @@ constexpr int QUERY_TILE = 128;       // tcgen05 path: queries per CTA (MMA M)
 constexpr int ROW_TILE = 256;         // tcgen05 path: cache rows per accumulator (MMA N)
 constexpr int K_CHUNK = 64;           // tcgen05 path: bf16 elements per 128-byte swizzled row
 constexpr int UMMA_STAGE_BYTES = (QUERY_TILE + ROW_TILE) * K_CHUNK * 2;  // 48 KiB
-constexpr int SCAN_MAX_Q = 4;
+constexpr int SCAN_MAX_Q = 4;        // queries per scan launch
+constexpr int SCAN_AUTO_MAX_Q = 2;   // largest batch the automatic choice gives to the scan path
 constexpr int SCAN_MAX_DIM = 1024;
 constexpr int SCAN_ROWS_PER_STAGE = 32;
 constexpr int SCAN_CONSUMER_WARPS = 8;
@@ -160,7 +161,9 @@ int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32
   if (path < IC_PATH_AUTO || path > IC_PATH_UMMA) return fail(IC_ERR_INVALID, "plan: unknown path %d", path);
   const int window = std::min<int>(nq, WINDOW_MAX_NQ);
   const int n_windows = (nq + WINDOW_MAX_NQ - 1) / WINDOW_MAX_NQ;
-  if (path == IC_PATH_AUTO) path = (nq <= SCAN_MAX_Q && dim <= SCAN_MAX_DIM) ? IC_PATH_SCAN : IC_PATH_UMMA;
+  // measured crossover (N = 1 M, d = 768, k = 10): the scan wins for one or two queries, the
+  // tensor-core path from three on (its time hardly grows with nq while HBM-bound)
+  if (path == IC_PATH_AUTO) path = (nq <= SCAN_AUTO_MAX_Q && dim <= SCAN_MAX_DIM) ? IC_PATH_SCAN : IC_PATH_UMMA;
   out->path = path;
   const int merge_lists_max = (smem_optin - 4096) / (k * 8 + 4);
   if (path == IC_PATH_GENERIC) {
@@ -198,7 +201,9 @@ int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32
     // Threshold seeding: with enough row tiles per CTA, first score 1/16 of them, merge that
     // sample's lists into its exact top-k and start the main pass from the sample's k-th key.
     const int64_t n_tiles = (n + ROW_TILE - 1) / ROW_TILE;
-    if (n_tiles >= (int64_t)SEED_MIN_TILES_PER_CTA * out->n_partitions) {
+    const char* seed_env = getenv("IC_CACHE_SEED");   // tuning knob: "0" scores everything in one pass
+    const bool seeding = !(seed_env && seed_env[0] == '0' && seed_env[1] == 0);
+    if (seeding && n_tiles >= (int64_t)SEED_MIN_TILES_PER_CTA * out->n_partitions) {
       const int64_t t = n_tiles / SEED_FRACTION / out->n_partitions * out->n_partitions;
       out->seed_tiles = (int32_t)std::max<int64_t>(out->n_partitions, t);
       // with several tiles per CTA in that sample, seed the sample itself from one tile per CTA
@@ -244,12 +249,10 @@ int check_timeout(ic_cache* c) {
 
 int do_insert(ic_cache* c, const void* emb, const int64_t* ids, int64_t n) {
   cudaError_t e = icc::launch_convert_rows(emb, c->input_dtype == IC_F32, n, c->dim, c->normalize,
-                                           static_cast<char*>(c->slab) + (size_t)c->size * c->dim * 2, nullptr, n,
-                                           c->stream);
+                                           static_cast<char*>(c->slab) + (size_t)c->size * c->dim * 2, nullptr, n, ids,
+                                           c->ids + c->size, c->stream);
   if (e != cudaSuccess) return fail(IC_ERR_CUDA, "insert kernel launch failed: %s", cudaGetErrorString(e));
   c->launches += 1;
-  e = cudaMemcpyAsync(c->ids + c->size, ids, (size_t)n * 8, cudaMemcpyDeviceToDevice, c->stream);
-  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "id copy failed: %s", cudaGetErrorString(e));
   c->size += n;
   return IC_OK;
 }
@@ -347,7 +350,7 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
   if ((rc = ensure(c, c->thr, (size_t)nq * 8, "seed thresholds")) != IC_OK) return rc;
 
   cudaError_t e = icc::launch_convert_rows(q, c->input_dtype == IC_F32, nq, c->dim, c->normalize, c->q_bf16.p,
-                                           static_cast<float*>(c->q_f32.p), nq_pad, c->stream);
+                                           static_cast<float*>(c->q_f32.p), nq_pad, nullptr, nullptr, c->stream);
   if (e != cudaSuccess) return fail(IC_ERR_CUDA, "query preparation launch failed: %s", cudaGetErrorString(e));
   c->launches += 1;
   uint64_t* partials = static_cast<uint64_t*>(c->partials.p);
@@ -449,7 +452,7 @@ int do_query_window_static(ic_cache* c, const void* q, int nq, int k, int64_t* o
   unsigned long long* pace = reinterpret_cast<unsigned long long*>(base + off_pace);
 
   cudaError_t e = icc::launch_convert_rows(q, c->input_dtype == IC_F32, nq, c->dim, c->normalize, q_bf16, q_f32, nq_pad,
-                                           c->stream);
+                                           nullptr, nullptr, c->stream);
   if (e != cudaSuccess) return fail(IC_ERR_CUDA, "query preparation launch failed: %s", cudaGetErrorString(e));
   c->launches += 1;
   int n_final_lists = pl.n_partitions;

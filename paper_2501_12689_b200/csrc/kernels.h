@@ -6,11 +6,40 @@
 
 namespace icc {
 
+// Launch `kernel` so that it may overlap the tail of the previous kernel in the stream
+// (programmatic stream serialisation); cluster_x > 1 also asks for thread-block clusters.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                     int cluster_x, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cluster_x > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = (unsigned)cluster_x;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = (unsigned)n;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Convert/normalise `nrows` input rows ([nrows, dim], fp32 if in_is_f32 else bf16) into bf16
 // rows at out_bf16 (row pitch = dim elements).  Rows nrows .. pad_rows-1 of out_bf16 are set
 // to zero.  If out_f32 != NULL it receives the stored bf16 values widened to fp32.
+// ids_in/ids_out: optional, copies one int64 label per row alongside (used by insert).
 cudaError_t launch_convert_rows(const void* in, int in_is_f32, int64_t nrows, int dim, int normalize,
-                                void* out_bf16, float* out_f32, int64_t pad_rows, cudaStream_t st);
+                                void* out_bf16, float* out_f32, int64_t pad_rows, const int64_t* ids_in,
+                                int64_t* ids_out, cudaStream_t st);
 
 // Generic CUDA-core scoring of up to 4 queries [q0, q0+4) against rows [0, n).
 // partials: [n_part][nq][k] packed keys.

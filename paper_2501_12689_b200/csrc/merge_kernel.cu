@@ -6,6 +6,7 @@
 
 #include "common.cuh"
 #include "kernels.h"
+#include "pipeline.cuh"
 
 namespace icc {
 
@@ -54,6 +55,8 @@ merge_topk_kernel(const uint64_t* __restrict__ partials, int n_part, int nq, int
 
   const int q = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
   const int total = n_part * k;
+  grid_dep_launch_dependents();
+  grid_dep_wait();   // the partial lists come from the previous kernel
   // list p of this query is k contiguous keys at partials[(p * nq + q) * k]; several loads
   // per thread are in flight at once
 #pragma unroll 4
@@ -100,18 +103,16 @@ cudaError_t launch_merge(const uint64_t* partials, int n_part, int nq, int k, co
                          int64_t* out_ids, float* out_scores, cudaStream_t st) {
   const size_t smem = (size_t)n_part * k * 8 + (size_t)n_part * 4;
   if (smem > (size_t)g_merge_smem_limit) return cudaErrorInvalidValue;
-  merge_topk_kernel<<<nq, MERGE_THREADS, smem, st>>>(partials, n_part, nq, k, ids, out_ids, out_scores, nullptr,
-                                                     nullptr);
-  return cudaGetLastError();
+  return launch_overlapped(merge_topk_kernel, dim3(nq), dim3(MERGE_THREADS), smem, st, 1, partials, n_part, nq, k, ids,
+                           out_ids, out_scores, (uint64_t*)nullptr, (uint64_t*)nullptr);
 }
 
 cudaError_t launch_merge_keys(const uint64_t* partials, int n_part, int nq, int k, uint64_t* out_keys,
                               uint64_t* out_thr, cudaStream_t st) {
   const size_t smem = (size_t)n_part * k * 8 + (size_t)n_part * 4;
   if (smem > (size_t)g_merge_smem_limit || !out_keys || !out_thr) return cudaErrorInvalidValue;
-  merge_topk_kernel<<<nq, MERGE_THREADS, smem, st>>>(partials, n_part, nq, k, nullptr, nullptr, nullptr, out_keys,
-                                                     out_thr);
-  return cudaGetLastError();
+  return launch_overlapped(merge_topk_kernel, dim3(nq), dim3(MERGE_THREADS), smem, st, 1, partials, n_part, nq, k,
+                           (const int64_t*)nullptr, (int64_t*)nullptr, (float*)nullptr, out_keys, out_thr);
 }
 
 }  // namespace icc

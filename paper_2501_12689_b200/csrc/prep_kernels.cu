@@ -2,6 +2,7 @@
 // staging buffers): optional fp32 L2 normalisation, then round-to-nearest-even to bf16.
 #include "common.cuh"
 #include "kernels.h"
+#include "pipeline.cuh"
 
 namespace icc {
 
@@ -13,7 +14,9 @@ template <bool IN_F32>
 __global__ void __launch_bounds__(CONV_WARPS * 32)
 convert_rows_kernel(const void* __restrict__ in, int64_t nrows, int dim, int normalize,
                     __nv_bfloat16* __restrict__ out_bf16, float* __restrict__ out_f32,
-                    int64_t pad_rows) {
+                    int64_t pad_rows, const int64_t* __restrict__ ids_in, int64_t* __restrict__ ids_out) {
+  grid_dep_launch_dependents();
+  grid_dep_wait();   // the destination may still be read by the previous kernel in the stream
   const int lane = threadIdx.x & 31;
   const int64_t row = (int64_t)blockIdx.x * CONV_WARPS + (threadIdx.x >> 5);
   if (row >= pad_rows) return;
@@ -23,6 +26,7 @@ convert_rows_kernel(const void* __restrict__ in, int64_t nrows, int dim, int nor
     for (int c = lane; c < nchunk; c += 32) orow[c] = make_uint4(0, 0, 0, 0);
     return;
   }
+  if (ids_in && lane == 0) ids_out[row] = ids_in[row];
   float x[CONV_MAX_CHUNKS / 1][8];
   float ss = 0.0f;
 #pragma unroll
@@ -73,17 +77,16 @@ convert_rows_kernel(const void* __restrict__ in, int64_t nrows, int dim, int nor
 }
 
 cudaError_t launch_convert_rows(const void* in, int in_is_f32, int64_t nrows, int dim, int normalize,
-                                void* out_bf16, float* out_f32, int64_t pad_rows, cudaStream_t st) {
+                                void* out_bf16, float* out_f32, int64_t pad_rows, const int64_t* ids_in,
+                                int64_t* ids_out, cudaStream_t st) {
   if (pad_rows < nrows) pad_rows = nrows;
   if (pad_rows == 0) return cudaSuccess;
   const unsigned blocks = (unsigned)((pad_rows + CONV_WARPS - 1) / CONV_WARPS);
   if (in_is_f32)
-    convert_rows_kernel<true><<<blocks, CONV_WARPS * 32, 0, st>>>(
-        in, nrows, dim, normalize, static_cast<__nv_bfloat16*>(out_bf16), out_f32, pad_rows);
-  else
-    convert_rows_kernel<false><<<blocks, CONV_WARPS * 32, 0, st>>>(
-        in, nrows, dim, normalize, static_cast<__nv_bfloat16*>(out_bf16), out_f32, pad_rows);
-  return cudaGetLastError();
+    return launch_overlapped(convert_rows_kernel<true>, dim3(blocks), dim3(CONV_WARPS * 32), 0, st, 1, in, nrows, dim,
+                             normalize, static_cast<__nv_bfloat16*>(out_bf16), out_f32, pad_rows, ids_in, ids_out);
+  return launch_overlapped(convert_rows_kernel<false>, dim3(blocks), dim3(CONV_WARPS * 32), 0, st, 1, in, nrows, dim,
+                           normalize, static_cast<__nv_bfloat16*>(out_bf16), out_f32, pad_rows, ids_in, ids_out);
 }
 
 }  // namespace icc

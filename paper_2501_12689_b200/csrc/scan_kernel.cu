@@ -70,6 +70,8 @@ scan_score_topk_kernel(const __nv_bfloat16* __restrict__ slab, int64_t n, int di
     mbar_fence_init();
   }
   for (int i = tid; i < SCAN_CONSUMER_WARPS * SCAN_MAX_QB * k; i += SCAN_THREADS) lists[i] = KEY_EMPTY;
+  grid_dep_launch_dependents();
+  grid_dep_wait();   // queries and newly inserted rows come from earlier kernels in the stream
   __syncthreads();
 
   const int64_t n_pieces = (n + SCAN_STAGE_ROWS - 1) / SCAN_STAGE_ROWS;
@@ -190,10 +192,9 @@ scan_score_topk_kernel(const __nv_bfloat16* __restrict__ slab, int64_t n, int di
 
 template <int QB, int NCHUNK>
 static cudaError_t launch_scan_t(const ScanParams& p, cudaStream_t st) {
-  scan_score_topk_kernel<QB, NCHUNK><<<p.n_part, SCAN_THREADS, p.smem_bytes, st>>>(
-      static_cast<const __nv_bfloat16*>(p.slab), p.n, p.dim, p.q_f32, p.q0, p.nq, p.k, p.partials, p.n_stages,
-      p.dev_status);
-  return cudaGetLastError();
+  return launch_overlapped(scan_score_topk_kernel<QB, NCHUNK>, dim3(p.n_part), dim3(SCAN_THREADS), (size_t)p.smem_bytes,
+                           st, 1, static_cast<const __nv_bfloat16*>(p.slab), p.n, p.dim, p.q_f32, p.q0, p.nq, p.k,
+                           p.partials, p.n_stages, p.dev_status);
 }
 
 template <int QB>

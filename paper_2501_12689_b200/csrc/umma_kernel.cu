@@ -97,6 +97,8 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     if (CG == 2) tmem_alloc_pair(&tail->tmem_base, UM_TMEM_COLS);
     else tmem_alloc(&tail->tmem_base, UM_TMEM_COLS);
   }
+  grid_dep_launch_dependents();
+  grid_dep_wait();   // queries, thresholds and new rows come from earlier kernels in the stream
   tc_fence_before_sync();
   __syncthreads();
   if (CG == 2) cluster_sync_all();   // the peer's barriers are initialised before anyone signals them
@@ -454,27 +456,16 @@ cudaError_t launch_umma(const UmmaParams& p, cudaStream_t st) {
   const int stage_bytes = p.cta_group == 2 ? um_stage_bytes<2>() : um_stage_bytes<1>();
   const size_t need = 1024 + (size_t)p.n_stages * stage_bytes + (size_t)UM_QT * (p.k + p.queue_cap) * 8 + sizeof(UmmaSmemTail);
   if (need > (size_t)p.smem_bytes) return cudaErrorInvalidValue;
-  cudaLaunchConfig_t cfg;
-  memset(&cfg, 0, sizeof cfg);
-  cfg.gridDim = dim3((unsigned)(p.n_part * p.n_query_tiles), 1, 1);
-  cfg.blockDim = dim3(UM_THREADS, 1, 1);
-  cfg.dynamicSmemBytes = (size_t)p.smem_bytes;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  if (p.cta_group == 2) {
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, umma_score_topk_kernel<2>, p.tmap_q, p.tmap_slab_half, p.n, p.tile_begin, p.tile_end,
-                              p.dim, p.nq, p.k, p.n_query_tiles, p.n_part, p.n_stages, p.queue_cap, p.thr_floor,
-                              p.partials, p.pace, p.pace_epoch, p.pace_window, p.dev_status);
-  }
-  return cudaLaunchKernelEx(&cfg, umma_score_topk_kernel<1>, p.tmap_q, p.tmap_slab, p.n, p.tile_begin, p.tile_end, p.dim,
-                            p.nq, p.k, p.n_query_tiles, p.n_part, p.n_stages, p.queue_cap, p.thr_floor, p.partials,
-                            p.pace, p.pace_epoch, p.pace_window, p.dev_status);
+  const dim3 grid((unsigned)(p.n_part * p.n_query_tiles));
+  if (p.cta_group == 2)
+    return launch_overlapped(umma_score_topk_kernel<2>, grid, dim3(UM_THREADS), (size_t)p.smem_bytes, st, 2, p.tmap_q,
+                             p.tmap_slab_half, p.n, p.tile_begin, p.tile_end, p.dim, p.nq, p.k, p.n_query_tiles, p.n_part,
+                             p.n_stages, p.queue_cap, p.thr_floor, p.partials, p.pace, p.pace_epoch, p.pace_window,
+                             p.dev_status);
+  return launch_overlapped(umma_score_topk_kernel<1>, grid, dim3(UM_THREADS), (size_t)p.smem_bytes, st, 1, p.tmap_q,
+                           p.tmap_slab, p.n, p.tile_begin, p.tile_end, p.dim, p.nq, p.k, p.n_query_tiles, p.n_part,
+                           p.n_stages, p.queue_cap, p.thr_floor, p.partials, p.pace, p.pace_epoch, p.pace_window,
+                           p.dev_status);
 }
 
 }  // namespace icc

@@ -44,8 +44,11 @@ def test_header_constants_match_binding():
 def test_plan_paths_and_shapes():
     p = pkg.ic_cache_plan(768, 1_000_000, 1, 10)
     assert p["path"] == pkg.IC_PATH_SCAN and p["query_tile"] == 1 and p["n_ctas"] == 148 and p["n_stages"] >= 2
-    p = pkg.ic_cache_plan(768, 1_000_000, 4, 10)
-    assert p["path"] == pkg.IC_PATH_SCAN and p["query_tile"] == 4 and p["n_launches"] == 1
+    p = pkg.ic_cache_plan(768, 1_000_000, 2, 10)
+    assert p["path"] == pkg.IC_PATH_SCAN and p["query_tile"] == 2 and p["n_launches"] == 1
+    p = pkg.ic_cache_plan(768, 1_000_000, 4, 10, path=pkg.IC_PATH_SCAN)
+    assert p["query_tile"] == 4 and p["n_launches"] == 1
+    assert pkg.ic_cache_plan(768, 1_000_000, 4, 10)["path"] == pkg.IC_PATH_UMMA
     p = pkg.ic_cache_plan(768, 1_000_000, 64, 10)
     assert p["path"] == pkg.IC_PATH_UMMA and p["n_query_tiles"] == 1 and p["n_partitions"] == 148
     p = pkg.ic_cache_plan(1024, 4_000_000, 256, 32)
