@@ -30,6 +30,11 @@ if ROOT not in sys.path:
 METRIC = "retrieval_queries_per_sec"
 UNIT = "queries/s"
 
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the ncu
+# captures summarised under profiles/ (key: workload, rows, nq).  An entry is removed (the JSON
+# then says null) whenever that kernel changes after its capture.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+
 
 def parse_args():
     ap = argparse.ArgumentParser()
@@ -277,32 +282,41 @@ def run_ours(args):
         return
 
     def roofline_of(r):
-        """Roofline of the scoring kernel (the fused score + partial top-k launch).
-        Algorithmic bytes = 2*dim per cache row per launch (each launch reads the slab once);
-        flops = 2*dim per (query, row) pair.  The bound is whichever takes longer at the peaks."""
+        """Roofline of the dominant kernel: the main scoring launch (fused score + partial top-k;
+        on the tensor-core path the launch that reads every row outside the seeding samples).
+        Algorithmic bytes per launch = 2*dim per row it scans, flops = 2*dim per (query, row);
+        the bound is whichever takes longer at the measured peaks."""
         pr = r["profile"]
         if not pr or pr["scoring_launches"] == 0:
             return None
-        rows = r["rows_scanned"] / r["steps"]                     # mean rows per step
+        rows = r["rows_scanned"] / r["steps"]                     # mean cache rows per step
+        pl = ic_cache_plan(w.dim, int(rows), r["nq"], w.k, path, props.multi_processor_count,
+                           props.shared_memory_per_block_optin)
         launches_per_step = pr["scoring_launches"] / r["steps"]
-        bytes_per_launch = rows * w.dim * 2
-        flops_per_step = rows * w.dim * 2 * r["nq"]
+        rows_main = rows - min(rows, pl["seed_tiles"] * 256)       # rows the dominant launch reads
+        bytes_per_launch = rows_main * w.dim * 2
+        flops_per_launch = bytes_per_launch * min(r["nq"], pl["query_tile"] * pl["n_query_tiles"])
         t_launch = pr["scoring_ms"] * 1e-3 / pr["scoring_launches"]
-        t_hbm = bytes_per_launch * launches_per_step / (peaks["hbm_gbs"] * 1e9)
-        t_tensor = flops_per_step / (peaks["bf16_tflops_sustained"] * 1e12)
+        t_hbm = bytes_per_launch / (peaks["hbm_gbs"] * 1e9)
+        t_tensor = flops_per_launch / (peaks["bf16_tflops_sustained"] * 1e12)
         if t_hbm >= t_tensor:
             ach = bytes_per_launch / t_launch / 1e9
             out = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                    "frac": ach / peaks["hbm_gbs"]}
         else:
-            ach = flops_per_step / (t_launch * launches_per_step) / 1e12
+            ach = flops_per_launch / t_launch / 1e12
             out = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                    "frac": ach / peaks["bf16_tflops_sustained"]}
-        out.update({"traffic": None, "peak_source": peaks["source"], "kernel": "scoring + partial top-k",
+        traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH.get((w.name, w.n, r["nq"]))
+        out.update({"traffic": traffic, "peak_source": peaks["source"] + " (sustained figure for tensor)",
+                    "kernel": {2: "scan_score_topk_kernel", 3: "umma_score_topk_kernel (main pass)",
+                               1: "generic_score_topk_kernel"}[pl["path"]],
                     "kernel_us_per_launch": t_launch * 1e6,
-                    "merge_us_per_launch": pr["merge_ms"] * 1e3 / max(1, pr["merge_launches"]),
                     "launches_per_step": launches_per_step,
-                    "algorithmic_bytes_per_launch": bytes_per_launch})
+                    "algorithmic_bytes_per_launch": bytes_per_launch,
+                    "rows_per_launch": rows_main,
+                    "seed_passes_us_per_step": pr["seed_ms"] * 1e3 / r["steps"],
+                    "final_merge_us_per_step": pr["merge_ms"] * 1e3 / r["steps"]})
         return out
 
     plan = ic_cache_plan(w.dim, w.n, nq, w.k, path, props.multi_processor_count,

@@ -196,16 +196,20 @@ int ic_cache_sync(ic_cache_t* c);
 int64_t ic_cache_launch_count(const ic_cache_t* c);
 
 /*
- * Measurement aid.  While enabled, every scoring-kernel launch and every merge launch of this
- * handle is bracketed by a pair of CUDA events on the handle's stream (at most 16384 launches
- * of each kind between two reads; later ones go unrecorded).
+ * Measurement aid.  While enabled, the launches of this handle are bracketed by pairs of CUDA
+ * events on the handle's stream, in three groups: "scoring" = the scan launch(es), or the main
+ * pass of the tensor-core path (the launch that reads all rows outside the seeding samples);
+ * "seed" = each threshold-seeding pass together with the merge of its lists; "merge" = the
+ * final merge.  At most 16384 brackets of each group between two reads; later ones go
+ * unrecorded.  ic_cache_query_static records nothing.
  */
 int ic_cache_set_profiling(ic_cache_t* c, int32_t enable);
 
-/* Synchronise the stream and return the device time (ms) and number of the scoring and merge
- * launches recorded since the previous read.  Any output pointer may be NULL. */
+/* Synchronise the stream and return the device time (ms) and number of brackets of each group
+ * recorded since the previous read.  Any output pointer may be NULL. */
 int ic_cache_read_profile(ic_cache_t* c, double* scoring_ms, int64_t* scoring_launches,
-                          double* merge_ms, int64_t* merge_launches);
+                          double* merge_ms, int64_t* merge_launches, double* seed_ms,
+                          int64_t* seed_passes);
 
 /*
  * The launch plan the library would use for a query of nq vectors, k results, over n entries

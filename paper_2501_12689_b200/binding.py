@@ -77,6 +77,7 @@ SIGNATURES = {
     "ic_cache_set_profiling": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32]),
     "ic_cache_read_profile": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_double),
                                              ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
+                                             ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
                                              ctypes.POINTER(ctypes.c_int64)]),
     "ic_cache_plan": (ctypes.c_int, [ctypes.c_int32, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                      ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ic_cache_plan_t)]),
@@ -280,13 +281,16 @@ class ICCache:
         _check(load_library().ic_cache_set_profiling(self._h, int(bool(enable))))
 
     def read_profile(self) -> dict:
-        """Device time of the scoring and merge launches recorded since the last read."""
-        s_ms, m_ms = ctypes.c_double(), ctypes.c_double()
-        s_n, m_n = ctypes.c_int64(), ctypes.c_int64()
+        """Device time of the main scoring launches, the seeding passes (each with its merge) and
+        the final merges recorded since the last read."""
+        s_ms, m_ms, d_ms = ctypes.c_double(), ctypes.c_double(), ctypes.c_double()
+        s_n, m_n, d_n = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
         _check(load_library().ic_cache_read_profile(self._h, ctypes.byref(s_ms), ctypes.byref(s_n),
-                                                    ctypes.byref(m_ms), ctypes.byref(m_n)))
+                                                    ctypes.byref(m_ms), ctypes.byref(m_n),
+                                                    ctypes.byref(d_ms), ctypes.byref(d_n)))
         return {"scoring_ms": s_ms.value, "scoring_launches": s_n.value,
-                "merge_ms": m_ms.value, "merge_launches": m_n.value}
+                "merge_ms": m_ms.value, "merge_launches": m_n.value,
+                "seed_ms": d_ms.value, "seed_passes": d_n.value}
 
     @property
     def size(self) -> int:

@@ -94,8 +94,8 @@ struct ic_cache {
   bool have_tmap_slab = false;
   // optional per-kernel timing (ic_cache_set_profiling)
   bool profiling = false;
-  std::vector<cudaEvent_t> ev_score, ev_merge;   // start/stop pairs
-  size_t n_ev_score = 0, n_ev_merge = 0;         // events used since the last read
+  std::vector<cudaEvent_t> ev_score, ev_merge, ev_seed;   // start/stop pairs
+  size_t n_ev_score = 0, n_ev_merge = 0, n_ev_seed = 0;   // events used since the last read
 };
 
 namespace {
@@ -265,7 +265,8 @@ int do_insert(ic_cache* c, const void* emb, const int64_t* ids, int64_t n) {
 //   blocks P+1 .. 2P     lists of a seeding pass                block 2P+1   first sample's merged list
 // On return *n_final_lists tells the final merge how many leading blocks to read.
 int run_umma_passes(ic_cache* c, const ic_cache_plan_t& pl, const void* q_bf16, int nq, int nq_pad, int k,
-                    uint64_t* partials, uint64_t* thr, unsigned long long* pace, int* n_final_lists) {
+                    uint64_t* partials, uint64_t* thr, unsigned long long* pace, int* n_final_lists,
+                    bool profile) {
   if (!c->have_tmap_slab) return fail(IC_ERR_UNSUPPORTED, "tensor-core path unavailable: no tensor map for the slab");
   const int P = pl.n_partitions;
   const size_t list_block = (size_t)nq * k;
@@ -312,6 +313,7 @@ int run_umma_passes(ic_cache* c, const ic_cache_plan_t& pl, const void* q_bf16, 
     up.thr_floor = have_thr ? thr : nullptr;
     up.partials = pass_lists;
     up.pace_epoch = ++c->pace_epoch;
+    if (profile) profile_mark(c, c->ev_seed, c->n_ev_seed);
     cudaError_t e = icc::launch_umma(up, c->stream);
     if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core seeding launch failed: %s", cudaGetErrorString(e));
     c->launches += 1;
@@ -321,6 +323,7 @@ int run_umma_passes(ic_cache* c, const ic_cache_plan_t& pl, const void* q_bf16, 
                                c->stream);
     if (e != cudaSuccess) return fail(IC_ERR_CUDA, "seed merge launch failed: %s", cudaGetErrorString(e));
     c->launches += 1;
+    if (profile) profile_mark(c, c->ev_seed, c->n_ev_seed);
     have_thr = true;
     begin = end;
     *n_final_lists = P + 1;
@@ -330,9 +333,11 @@ int run_umma_passes(ic_cache* c, const ic_cache_plan_t& pl, const void* q_bf16, 
   up.thr_floor = have_thr ? thr : nullptr;
   up.partials = partials;
   up.pace_epoch = ++c->pace_epoch;
+  if (profile) profile_mark(c, c->ev_score, c->n_ev_score);
   cudaError_t e = icc::launch_umma(up, c->stream);
   if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core scoring launch failed: %s", cudaGetErrorString(e));
   c->launches += 1;
+  if (profile) profile_mark(c, c->ev_score, c->n_ev_score);
   return IC_OK;
 }
 
@@ -356,7 +361,7 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
   uint64_t* partials = static_cast<uint64_t*>(c->partials.p);
   int n_final_lists = pl.n_partitions;
 
-  profile_mark(c, c->ev_score, c->n_ev_score);
+  if (pl.path != IC_PATH_UMMA) profile_mark(c, c->ev_score, c->n_ev_score);
   if (pl.path == IC_PATH_GENERIC) {
     for (int q0 = 0; q0 < nq; q0 += GENERIC_QB) {
       e = icc::launch_generic(c->slab, c->size, c->dim, static_cast<const float*>(c->q_f32.p), q0, nq, k,
@@ -387,10 +392,10 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
     }
   } else {
     rc = run_umma_passes(c, pl, c->q_bf16.p, nq, nq_pad, k, partials, static_cast<uint64_t*>(c->thr.p),
-                         static_cast<unsigned long long*>(c->pace.p), &n_final_lists);
+                         static_cast<unsigned long long*>(c->pace.p), &n_final_lists, true);
     if (rc != IC_OK) return rc;
   }
-  profile_mark(c, c->ev_score, c->n_ev_score);
+  if (pl.path != IC_PATH_UMMA) profile_mark(c, c->ev_score, c->n_ev_score);
   profile_mark(c, c->ev_merge, c->n_ev_merge);
   e = icc::launch_merge(partials, n_final_lists, nq, k, c->ids, out_ids, out_scores, c->stream);
   if (e != cudaSuccess) return fail(IC_ERR_CUDA, "merge launch failed: %s", cudaGetErrorString(e));
@@ -485,7 +490,7 @@ int do_query_window_static(ic_cache* c, const void* q, int nq, int k, int64_t* o
       c->launches += 1;
     }
   } else {
-    rc = run_umma_passes(c, pl, q_bf16, nq, nq_pad, k, partials, thr, pace, &n_final_lists);
+    rc = run_umma_passes(c, pl, q_bf16, nq, nq_pad, k, partials, thr, pace, &n_final_lists, false);
     if (rc != IC_OK) return rc;
   }
   e = icc::launch_merge(partials, n_final_lists, nq, k, c->ids, out_ids, out_scores, c->stream);
@@ -694,6 +699,7 @@ void ic_cache_destroy(ic_cache_t* c) {
   if (c->h_status) cudaFreeHost(c->h_status);
   for (cudaEvent_t ev : c->ev_score) cudaEventDestroy(ev);
   for (cudaEvent_t ev : c->ev_merge) cudaEventDestroy(ev);
+  for (cudaEvent_t ev : c->ev_seed) cudaEventDestroy(ev);
   cudaGetLastError();
   delete c;
 }
@@ -856,16 +862,16 @@ int ic_cache_set_profiling(ic_cache_t* c, int32_t enable) {
 }
 
 int ic_cache_read_profile(ic_cache_t* c, double* scoring_ms, int64_t* scoring_launches, double* merge_ms,
-                          int64_t* merge_launches) {
+                          int64_t* merge_launches, double* seed_ms, int64_t* seed_passes) {
   if (!c) return fail(IC_ERR_INVALID, "NULL handle");
   DeviceGuard guard(c->device);
   cudaError_t e = cudaStreamSynchronize(c->stream);
   if (e != cudaSuccess) return fail(IC_ERR_CUDA, "stream sync failed: %s", cudaGetErrorString(e));
-  double sums[2] = {0.0, 0.0};
-  int64_t counts[2] = {0, 0};
-  std::vector<cudaEvent_t>* pools[2] = {&c->ev_score, &c->ev_merge};
-  size_t* used[2] = {&c->n_ev_score, &c->n_ev_merge};
-  for (int w = 0; w < 2; ++w) {
+  double sums[3] = {0.0, 0.0, 0.0};
+  int64_t counts[3] = {0, 0, 0};
+  std::vector<cudaEvent_t>* pools[3] = {&c->ev_score, &c->ev_merge, &c->ev_seed};
+  size_t* used[3] = {&c->n_ev_score, &c->n_ev_merge, &c->n_ev_seed};
+  for (int w = 0; w < 3; ++w) {
     for (size_t i = 0; i + 1 < *used[w]; i += 2) {
       float ms = 0.0f;
       if (cudaEventElapsedTime(&ms, (*pools[w])[i], (*pools[w])[i + 1]) == cudaSuccess) {
@@ -881,6 +887,8 @@ int ic_cache_read_profile(ic_cache_t* c, double* scoring_ms, int64_t* scoring_la
   if (scoring_launches) *scoring_launches = counts[0];
   if (merge_ms) *merge_ms = sums[1];
   if (merge_launches) *merge_launches = counts[1];
+  if (seed_ms) *seed_ms = sums[2];
+  if (seed_passes) *seed_passes = counts[2];
   return IC_OK;
 }
 

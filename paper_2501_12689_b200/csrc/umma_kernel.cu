@@ -291,32 +291,32 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       const int64_t row0 = tile * UM_RT;
       if (lt == 0 && thr_floor_in == nullptr && k <= 16 && row0 + UM_RT <= n) {
         // Cold start (empty lists, no seed threshold): read the tile once just to take the
-        // maximum of each group of 16 columns.  The k-th largest of the 16 group maxima is a
-        // safe floor - k different columns score at least that much - and only ~6 % of the
-        // columns pass it, instead of every column passing an empty list.
-        float m[16];
+        // maximum of each group of 8 columns.  The k-th largest of the 32 group maxima is a
+        // safe floor - k different columns score at least that much - and only a few percent
+        // of the columns pass it (about 12 of 256 for k = 10, 21 for k = 16), instead of every
+        // column passing an empty list.
+        float m[32];
 #pragma unroll
         for (int cb = 0; cb < UM_RT / 32; ++cb) {
           uint32_t v[32];
           tmem_ld_32x32(t_addr + (uint32_t)(cb * 32), v);
           tmem_ld_wait();
-          float a = __uint_as_float(v[0]), b = __uint_as_float(v[16]);
 #pragma unroll
-          for (int c = 1; c < 16; ++c) {
-            a = fmaxf(a, __uint_as_float(v[c]));
-            b = fmaxf(b, __uint_as_float(v[16 + c]));
+          for (int gq = 0; gq < 4; ++gq) {
+            float a = __uint_as_float(v[8 * gq]);
+#pragma unroll
+            for (int c = 1; c < 8; ++c) a = fmaxf(a, __uint_as_float(v[8 * gq + c]));
+            m[4 * cb + gq] = a;
           }
-          m[2 * cb] = a;
-          m[2 * cb + 1] = b;
         }
         // bitonic sorting network, descending, on registers
 #pragma unroll
-        for (int ls = 1; ls <= 4; ++ls) {
+        for (int ls = 1; ls <= 5; ++ls) {
 #pragma unroll
-          for (int lj = 3; lj >= 0; --lj) {
+          for (int lj = 4; lj >= 0; --lj) {
             if (lj < ls) {
 #pragma unroll
-              for (int i = 0; i < 16; ++i) {
+              for (int i = 0; i < 32; ++i) {
                 const int j = i ^ (1 << lj);
                 if (j > i) {
                   const bool desc = (i & (1 << ls)) == 0;
@@ -328,10 +328,10 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             }
           }
         }
-        // m is sorted descending: its k-th entry is the largest of the entries k-1 .. 15
+        // m is sorted descending: its k-th entry is the largest of the entries k-1 .. 31
         float tau = -INFINITY;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) tau = fmaxf(tau, i >= k - 1 ? m[i] : -INFINITY);
+        for (int i = 0; i < 32; ++i) tau = fmaxf(tau, i >= k - 1 ? m[i] : -INFINITY);
         if (real && tau == tau) {
           // admit every key whose score is >= tau: the smallest such key has slot word 0
           thr_floor = ((uint64_t)score_to_ord(tau) << 32) - 1;
