@@ -130,6 +130,19 @@ int ic_cache_query(ic_cache_t* c, const void* q, int32_t nq, int32_t k, int64_t*
                    float* out_scores);
 
 /*
+ * ic_cache_query that reports only entries whose score reaches min_score: the hit test of
+ * semantic caching (paper Sec. 2.2: reuse a cached response when the most similar request is
+ * similar enough; its evaluation's similarity-threshold baselines) and a similarity pre-filter
+ * in front of the utility threshold of Sec. 4.1.  Same arguments, order and padding as
+ * ic_cache_query; entries of the top-k scoring below min_score are returned as id -1, score
+ * -infinity.  out_counts: optional device array [nq] of int32 receiving how many entries
+ * each query kept (0 .. min(k, size)); NULL to skip.  min_score = -infinity keeps everything;
+ * NaN is IC_ERR_INVALID.
+ */
+int ic_cache_query_min_score(ic_cache_t* c, const void* q, int32_t nq, int32_t k, float min_score,
+                             int64_t* out_ids, float* out_scores, int32_t* out_counts);
+
+/*
  * ic_cache_query for callers whose buffers live in HOST memory (pinned memory makes the
  * copies asynchronous): copies q to the device, runs the query, copies both results back
  * and synchronises the stream before returning.

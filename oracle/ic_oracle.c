@@ -156,3 +156,28 @@ int ic_oracle_search(const void* X, int x_dtype, const int64_t* ids, int64_t n, 
   free(order);
   return 0;
 }
+
+/*
+ * Similarity-threshold filter on a search result (the hit test of semantic caching, paper
+ * Sec. 2.2, and a similarity pre-filter before the utility threshold of Sec. 4.1): every
+ * entry whose score is below min_score becomes (id -1, slot -1, score -inf); counts[q]
+ * (optional) receives how many entries of query q remain.  Plain definition, entry by entry.
+ */
+void ic_oracle_apply_min_score(int64_t* out_ids, float* out_scores, int64_t* out_slots, int32_t nq, int32_t k,
+                               float min_score, int32_t* counts) {
+  for (int32_t iq = 0; iq < nq; ++iq) {
+    int32_t kept = 0;
+    for (int32_t r = 0; r < k; ++r) {
+      size_t o = (size_t)iq * (size_t)k + (size_t)r;
+      int present = out_scores[o] > -INFINITY || (out_ids && out_ids[o] != -1);
+      if (present && out_scores[o] >= min_score) {
+        ++kept;
+      } else {
+        if (out_ids) out_ids[o] = -1;
+        if (out_slots) out_slots[o] = -1;
+        out_scores[o] = -INFINITY;
+      }
+    }
+    if (counts) counts[iq] = kept;
+  }
+}

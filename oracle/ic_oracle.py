@@ -58,6 +58,9 @@ def _load():
             ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
             ctypes.c_void_p,
         ]
+        lib.ic_oracle_apply_min_score.restype = None
+        lib.ic_oracle_apply_min_score.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32,
+                                                  ctypes.c_int32, ctypes.c_float, ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -101,12 +104,14 @@ def default_threads() -> int:
 
 
 def search(x, q, k: int, ids=None, normalize: bool = False, round_bf16: bool = False,
-           threads: int | None = None, want_all_scores: bool = False):
+           threads: int | None = None, want_all_scores: bool = False, min_score: float | None = None):
     """Exhaustive cosine/inner-product top-k of every query row against every cache row.
 
     x: [n, d] float32, or uint16 holding bf16 bits.  q: [nq, d] likewise.
     ids: optional int64 [n] labels (default: the slot number).
     round_bf16: round float32 inputs to bf16 first (what a bf16 store keeps).
+    min_score: if given, entries scoring below it are reported as absent and the result also
+    carries counts [nq] int32 (entries kept per query).
     Returns dict(ids [nq,k] int64, scores [nq,k] float32, slots [nq,k] int64,
     all_scores [nq,n] float32 or None).  Rows past min(k, n) are (-1, -inf, -1).
     """
@@ -138,4 +143,10 @@ def search(x, q, k: int, ids=None, normalize: bool = False, round_bf16: bool = F
     )
     if rc != 0:
         raise RuntimeError(f"ic_oracle_search failed with code {rc}")
-    return {"ids": out_ids, "scores": out_scores, "slots": out_slots, "all_scores": all_scores}
+    res = {"ids": out_ids, "scores": out_scores, "slots": out_slots, "all_scores": all_scores}
+    if min_score is not None:
+        counts = np.empty((nq,), dtype=np.int32)
+        lib.ic_oracle_apply_min_score(out_ids.ctypes.data, out_scores.ctypes.data, out_slots.ctypes.data, nq, k,
+                                      float(min_score), counts.ctypes.data)
+        res["counts"] = counts
+    return res

@@ -62,6 +62,8 @@ SIGNATURES = {
     "ic_cache_insert": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64]),
     "ic_cache_query": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
                                       ctypes.c_void_p, ctypes.c_void_p]),
+    "ic_cache_query_min_score": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
+                                                ctypes.c_float, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "ic_cache_query_static": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
                                              ctypes.c_void_p, ctypes.c_void_p]),
     "ic_cache_query_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
@@ -147,6 +149,12 @@ def ic_cache_insert(h, emb: torch.Tensor, ids: torch.Tensor, n: Optional[int] = 
 
 def ic_cache_query(h, q: torch.Tensor, nq: int, k: int, out_ids: torch.Tensor, out_scores: torch.Tensor) -> None:
     _check(load_library().ic_cache_query(h, _ptr(q), nq, k, _ptr(out_ids), _ptr(out_scores)))
+
+
+def ic_cache_query_min_score(h, q: torch.Tensor, nq: int, k: int, min_score: float, out_ids: torch.Tensor,
+                             out_scores: torch.Tensor, out_counts: Optional[torch.Tensor]) -> None:
+    _check(load_library().ic_cache_query_min_score(h, _ptr(q), nq, k, min_score, _ptr(out_ids), _ptr(out_scores),
+                                                   _ptr(out_counts)))
 
 
 def ic_cache_query_static(h, q: torch.Tensor, nq: int, k: int, out_ids: torch.Tensor, out_scores: torch.Tensor) -> None:
@@ -239,6 +247,16 @@ class ICCache:
             out_scores = torch.empty(nq, k, dtype=torch.float32, device=self.device)
         ic_cache_query(self._h, q, nq, k, out_ids, out_scores)
         return out_ids, out_scores
+
+    def query_min_score(self, q: torch.Tensor, k: int, min_score: float):
+        """Top-k restricted to entries scoring at least min_score; returns (ids, scores, counts)."""
+        self._check_rows(q, True, "q")
+        nq = q.shape[0]
+        out_ids = torch.empty(nq, k, dtype=torch.int64, device=self.device)
+        out_scores = torch.empty(nq, k, dtype=torch.float32, device=self.device)
+        counts = torch.empty(nq, dtype=torch.int32, device=self.device)
+        ic_cache_query_min_score(self._h, q, nq, k, float(min_score), out_ids, out_scores, counts)
+        return out_ids, out_scores, counts
 
     def query_static(self, q: torch.Tensor, k: int, out_ids: torch.Tensor, out_scores: torch.Tensor) -> None:
         """Allocation-free query: results go into the caller's preallocated device tensors and

@@ -3,6 +3,7 @@
 // kernels; nothing here touches embedding data on the CPU.
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
 #include <stdlib.h>
@@ -342,7 +343,8 @@ int run_umma_passes(ic_cache* c, const ic_cache_plan_t& pl, const void* q_bf16, 
 }
 
 // One window of at most WINDOW_MAX_NQ queries, all pointers on the device.
-int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids, float* out_scores) {
+int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids, float* out_scores, float min_score,
+                    int32_t* out_counts) {
   ic_cache_plan_t pl;
   int rc = plan_impl(c->dim, c->size, nq, k, c->forced_path, c->sm_count, c->smem_optin, &pl);
   if (rc != IC_OK) return rc;
@@ -397,7 +399,7 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
   }
   if (pl.path != IC_PATH_UMMA) profile_mark(c, c->ev_score, c->n_ev_score);
   profile_mark(c, c->ev_merge, c->n_ev_merge);
-  e = icc::launch_merge(partials, n_final_lists, nq, k, c->ids, out_ids, out_scores, c->stream);
+  e = icc::launch_merge(partials, n_final_lists, nq, k, c->ids, out_ids, out_scores, min_score, out_counts, c->stream);
   if (e != cudaSuccess) return fail(IC_ERR_CUDA, "merge launch failed: %s", cudaGetErrorString(e));
   c->launches += 1;
   profile_mark(c, c->ev_merge, c->n_ev_merge);
@@ -433,6 +435,8 @@ int static_scratch_address(int dev, unsigned char** out) {
 // One query window with all scratch taken from the static array.  Mirrors do_query_window
 // but never grows a buffer, creates an event or allocates in any other way.
 int do_query_window_static(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids, float* out_scores) {
+  const float min_score = -INFINITY;
+  int32_t* const out_counts = nullptr;
   ic_cache_plan_t pl;
   int rc = plan_impl(c->dim, c->size, nq, k, c->forced_path, c->sm_count, c->smem_optin, &pl);
   if (rc != IC_OK) return rc;
@@ -493,7 +497,7 @@ int do_query_window_static(ic_cache* c, const void* q, int nq, int k, int64_t* o
     rc = run_umma_passes(c, pl, q_bf16, nq, nq_pad, k, partials, thr, pace, &n_final_lists, false);
     if (rc != IC_OK) return rc;
   }
-  e = icc::launch_merge(partials, n_final_lists, nq, k, c->ids, out_ids, out_scores, c->stream);
+  e = icc::launch_merge(partials, n_final_lists, nq, k, c->ids, out_ids, out_scores, min_score, out_counts, c->stream);
   if (e != cudaSuccess) return fail(IC_ERR_CUDA, "merge launch failed: %s", cudaGetErrorString(e));
   c->launches += 1;
   return IC_OK;
@@ -763,9 +767,17 @@ int ic_cache_insert_host(ic_cache_t* c, const void* emb_host, const int64_t* ids
 }
 
 int ic_cache_query(ic_cache_t* c, const void* q, int32_t nq, int32_t k, int64_t* out_ids, float* out_scores) {
+  return ic_cache_query_min_score(c, q, nq, k, -INFINITY, out_ids, out_scores, nullptr);
+}
+
+int ic_cache_query_min_score(ic_cache_t* c, const void* q, int32_t nq, int32_t k, float min_score, int64_t* out_ids,
+                             float* out_scores, int32_t* out_counts) {
   int rc = check_query_args(c, q, nq, k, out_ids, out_scores);
   if (rc != IC_OK || nq == 0) return rc;
+  if (min_score != min_score) return fail(IC_ERR_INVALID, "min_score is NaN");
   DeviceGuard guard(c->device);
+  if (out_counts && !is_device_ptr(out_counts, c->device))
+    return fail(IC_ERR_INVALID, "out_counts must be a device pointer on device %d", c->device);
   if (!is_device_ptr(q, c->device) || !is_device_ptr(out_ids, c->device) || !is_device_ptr(out_scores, c->device))
     return fail(IC_ERR_INVALID, "q, out_ids and out_scores must be device pointers on device %d (use ic_cache_query_host for host memory)", c->device);
   if ((rc = check_timeout(c)) != IC_OK) return rc;
@@ -773,7 +785,7 @@ int ic_cache_query(ic_cache_t* c, const void* q, int32_t nq, int32_t k, int64_t*
   for (int q0 = 0; q0 < nq; q0 += WINDOW_MAX_NQ) {
     const int w = std::min(WINDOW_MAX_NQ, nq - q0);
     rc = do_query_window(c, static_cast<const char*>(q) + (size_t)q0 * q_row, w, k, out_ids + (size_t)q0 * k,
-                         out_scores + (size_t)q0 * k);
+                         out_scores + (size_t)q0 * k, min_score, out_counts ? out_counts + q0 : nullptr);
     if (rc != IC_OK) return rc;
   }
   return IC_OK;
@@ -807,7 +819,7 @@ int ic_cache_query_host(ic_cache_t* c, const void* q_host, int32_t nq, int32_t k
     const int w = std::min(WINDOW_MAX_NQ, nq - q0);
     rc = do_query_window(c, static_cast<const char*>(c->stage_in.p) + (size_t)q0 * q_row, w, k,
                          static_cast<int64_t*>(c->stage_ids.p) + (size_t)q0 * k,
-                         static_cast<float*>(c->stage_scores.p) + (size_t)q0 * k);
+                         static_cast<float*>(c->stage_scores.p) + (size_t)q0 * k, -INFINITY, nullptr);
     if (rc != IC_OK) return rc;
   }
   e = cudaMemcpyAsync(out_ids_host, c->stage_ids.p, (size_t)nq * k * 8, cudaMemcpyDeviceToHost, c->stream);

@@ -89,9 +89,12 @@ struct UmmaParams {
 cudaError_t launch_umma(const UmmaParams& p, cudaStream_t st);
 cudaError_t umma_configure(int smem_optin);
 
-// Merge n_part partial lists per query into the final sorted top-k and gather ids.
+// Merge n_part partial lists per query into the final sorted top-k and gather ids.  Entries
+// scoring below min_score (-inf: none) are reported as absent; out_counts (optional, [nq])
+// receives the number of entries kept per query.
 cudaError_t launch_merge(const uint64_t* partials, int n_part, int nq, int k, const int64_t* ids,
-                         int64_t* out_ids, float* out_scores, cudaStream_t st);
+                         int64_t* out_ids, float* out_scores, float min_score, int32_t* out_counts,
+                         cudaStream_t st);
 // Same merge, but the result stays in key form: out_keys [nq][k] (sorted, KEY_EMPTY padded)
 // and out_thr [nq] = the k-th key (KEY_EMPTY when fewer than k candidates exist).
 cudaError_t launch_merge_keys(const uint64_t* partials, int n_part, int nq, int k, uint64_t* out_keys,

@@ -47,7 +47,7 @@ __global__ void __launch_bounds__(MERGE_THREADS)
 merge_topk_kernel(const uint64_t* __restrict__ partials, int n_part, int nq, int k,
                   const int64_t* __restrict__ ids, int64_t* __restrict__ out_ids,
                   float* __restrict__ out_scores, uint64_t* __restrict__ out_keys,
-                  uint64_t* __restrict__ out_thr) {
+                  uint64_t* __restrict__ out_thr, float min_score, int32_t* __restrict__ out_counts) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint64_t* cand = reinterpret_cast<uint64_t*>(smem_raw);                 // [n_part][k]
   uint32_t* pos = reinterpret_cast<uint32_t*>(cand + (size_t)n_part * k);  // [n_part]
@@ -83,10 +83,26 @@ merge_topk_kernel(const uint64_t* __restrict__ partials, int n_part, int nq, int
     if (tid == 0) out_thr[q] = win_key[k - 1];
     return;
   }
+  // Entries below min_score (-inf = keep all) are reported as absent; the list is sorted, so
+  // the kept entries are a prefix and their number is the query's hit count.
+  int kept = 0;
   for (int i = tid; i < k; i += MERGE_THREADS) {
     const uint64_t key = win_key[i];
-    out_scores[(size_t)q * k + i] = (key == KEY_EMPTY) ? -INFINITY : key_score(key);
-    out_ids[(size_t)q * k + i] = (key == KEY_EMPTY) ? (int64_t)-1 : ids[key_slot(key)];
+    const bool keep = (key != KEY_EMPTY) && (key_score(key) >= min_score);
+    out_scores[(size_t)q * k + i] = keep ? key_score(key) : -INFINITY;
+    out_ids[(size_t)q * k + i] = keep ? ids[key_slot(key)] : (int64_t)-1;
+    kept += keep ? 1 : 0;
+  }
+  if (out_counts) {
+    const int total_kept = __reduce_add_sync(FULL_MASK, kept);   // per warp
+    __shared__ int warp_kept[MERGE_THREADS / 32];
+    if (lane == 0) warp_kept[tid >> 5] = total_kept;
+    __syncthreads();
+    if (tid == 0) {
+      int sum = 0;
+      for (int w2 = 0; w2 < MERGE_THREADS / 32; ++w2) sum += warp_kept[w2];
+      out_counts[q] = sum;
+    }
   }
 }
 
@@ -100,11 +116,12 @@ cudaError_t merge_configure(int smem_optin) {
 }
 
 cudaError_t launch_merge(const uint64_t* partials, int n_part, int nq, int k, const int64_t* ids,
-                         int64_t* out_ids, float* out_scores, cudaStream_t st) {
+                         int64_t* out_ids, float* out_scores, float min_score, int32_t* out_counts,
+                         cudaStream_t st) {
   const size_t smem = (size_t)n_part * k * 8 + (size_t)n_part * 4;
   if (smem > (size_t)g_merge_smem_limit) return cudaErrorInvalidValue;
   return launch_overlapped(merge_topk_kernel, dim3(nq), dim3(MERGE_THREADS), smem, st, 1, partials, n_part, nq, k, ids,
-                           out_ids, out_scores, (uint64_t*)nullptr, (uint64_t*)nullptr);
+                           out_ids, out_scores, (uint64_t*)nullptr, (uint64_t*)nullptr, min_score, out_counts);
 }
 
 cudaError_t launch_merge_keys(const uint64_t* partials, int n_part, int nq, int k, uint64_t* out_keys,
@@ -112,7 +129,8 @@ cudaError_t launch_merge_keys(const uint64_t* partials, int n_part, int nq, int 
   const size_t smem = (size_t)n_part * k * 8 + (size_t)n_part * 4;
   if (smem > (size_t)g_merge_smem_limit || !out_keys || !out_thr) return cudaErrorInvalidValue;
   return launch_overlapped(merge_topk_kernel, dim3(nq), dim3(MERGE_THREADS), smem, st, 1, partials, n_part, nq, k,
-                           (const int64_t*)nullptr, (int64_t*)nullptr, (float*)nullptr, out_keys, out_thr);
+                           (const int64_t*)nullptr, (int64_t*)nullptr, (float*)nullptr, out_keys, out_thr, -INFINITY,
+                           (int32_t*)nullptr);
 }
 
 }  // namespace icc

@@ -236,3 +236,35 @@ def test_error_returns_leave_the_cache_unchanged():
     for dim, cap in ((0, 10), (12, 10), (8192, 10), (64, 0)):
         with pytest.raises(ICCacheError):
             ICCache(dim, cap)
+
+
+@pytest.mark.parametrize("path", ["generic", "scan", "umma"])
+def test_min_score_filter_and_counts(path):
+    w = wl.WORKLOADS["clustered"].scaled(50_000)
+    x = wl.cache_rows(w, DEV)
+    nq = 4 if path != "umma" else 40
+    q = wl.queries(w, nq, DEV, cache=x)
+    lab = wl.labels(w.n, DEV)
+    with ICCache(w.dim, w.n) as c:
+        c.set_path(PATHS[path])
+        c.insert(x, lab)
+        for tau in (0.85, 0.999, 2.0, float("-inf")):
+            ids, sc, counts = c.query_min_score(q, w.k, tau)
+            c.sync()
+            ref = oracle.search(wl.as_bits(x), wl.as_bits(q), w.k, ids=lab.cpu().numpy(), min_score=tau,
+                                want_all_scores=True)
+            got_counts = counts.cpu().numpy()
+            # a score within rounding distance of the threshold may fall on either side
+            near = np.abs(ref["all_scores"] - tau).min(axis=1) < 1e-5 if np.isfinite(tau) else np.zeros(nq, bool)
+            assert np.array_equal(got_counts[~near], ref["counts"][~near])
+            scn, idn = sc.cpu().numpy(), ids.cpu().numpy()
+            for i in range(nq):
+                kept = int(got_counts[i])
+                assert np.all(scn[i, :kept] >= tau) and np.all(np.isneginf(scn[i, kept:])) and np.all(idn[i, kept:] == -1)
+                if not near[i]:
+                    assert np.array_equal(idn[i, :kept], ref["ids"][i, :kept]) or \
+                        np.allclose(scn[i, :kept], ref["scores"][i, :kept], atol=1e-5)
+        assert counts.max().item() <= w.k
+    with ICCache(w.dim, 10) as c:
+        with pytest.raises(ICCacheError):
+            c.query_min_score(q, 3, float("nan"))

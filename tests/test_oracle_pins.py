@@ -298,3 +298,21 @@ def test_acceptance_rule_catches_planted_mistakes():
     accept(rl["ids"], rl["scores"], r["all_scores"], k, ids=lab, tol=1e-4)
     with pytest.raises(AcceptanceError):
         accept(r["ids"], r["scores"], r["all_scores"], k, ids=lab, tol=1e-4)
+
+
+# ---------------------------------------------------------------- similarity threshold
+
+def test_min_score_filter_hand_computed():
+    c = _parse_golden()["axes"]
+    x = np.array(c["x"], dtype=np.float32)
+    q = np.array([[1, 0], [0, 1], [0.6, 0.8]], dtype=np.float32)
+    r = oracle.search(x, q, k=4, min_score=0.7)
+    # from the golden file: q0 -> 0:1, 4:0.8 | q1 -> 1:1, 3:0.8 | q2 -> 3:1, 1:0.8 (0.6 and below drop)
+    assert r["counts"].tolist() == [2, 2, 2]
+    assert r["slots"].tolist() == [[0, 4, -1, -1], [1, 3, -1, -1], [3, 1, -1, -1]]
+    assert np.all(np.isneginf(r["scores"][:, 2:]))
+    np.testing.assert_allclose(r["scores"][:, :2], [[1, 0.8], [1, 0.8], [1, 0.8]], atol=1e-6)
+    # a threshold exactly at a score keeps it; above every score keeps nothing; -inf keeps all
+    assert oracle.search(x, q[:1], k=5, min_score=1.0)["counts"].tolist() == [1]
+    assert oracle.search(x, q[:1], k=5, min_score=1.5)["counts"].tolist() == [0]
+    assert oracle.search(x, q[:1], k=7, min_score=-np.inf)["counts"].tolist() == [5]
