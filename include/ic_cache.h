@@ -184,6 +184,20 @@ int ic_cache_query_static(ic_cache_t* c, const void* q, int32_t nq, int32_t k, i
 /* ic_cache_insert for HOST buffers; synchronises the stream before returning. */
 int ic_cache_insert_host(ic_cache_t* c, const void* emb_host, const int64_t* ids_host, int64_t n);
 
+/*
+ * Eviction mechanics (paper Sec. 4.3, "Example Manager": a background solver picks the
+ * examples to drop when the cache is full; which ones is the caller's policy).  Removes every
+ * entry whose id equals one of ids_host[0..n) (HOST array; ids that match nothing are
+ * ignored) and closes the gaps: surviving entries from the end of the slab move, in order,
+ * into the vacated slots, so size shrinks by the number removed and capacity is free again
+ * for ic_cache_insert.  After a removal "equal scores are ordered by earlier insertion"
+ * reads "by lower slot": a moved entry ranks among equal scores by its new position.
+ * *n_removed (optional) receives the number of entries removed.  Synchronises the stream.
+ * Not part of the per-request path: one pass over the id array (8 bytes per entry) plus the
+ * moved rows.  IC_ERR_UNSUPPORTED if more than 4n + 1024 entries carry the given ids.
+ */
+int ic_cache_remove(ic_cache_t* c, const int64_t* ids_host, int64_t n, int64_t* n_removed);
+
 /* Release the handle and everything the library allocated for it.  NULL is a no-op. */
 void ic_cache_destroy(ic_cache_t* c);
 

@@ -69,6 +69,7 @@ SIGNATURES = {
     "ic_cache_query_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
                                            ctypes.c_void_p, ctypes.c_void_p]),
     "ic_cache_insert_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64]),
+    "ic_cache_remove": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.POINTER(ctypes.c_int64)]),
     "ic_cache_destroy": (None, [ctypes.c_void_p]),
     "ic_cache_set_stream": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
     "ic_cache_set_path": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32]),
@@ -282,6 +283,14 @@ class ICCache:
             out_scores = torch.empty(nq, k, dtype=torch.float32).pin_memory()
         ic_cache_query_host(self._h, q, nq, k, out_ids, out_scores)
         return out_ids, out_scores
+
+    def remove(self, ids: torch.Tensor) -> int:
+        """Remove every entry whose id is in `ids` (a host int64 tensor); returns how many went."""
+        if ids.dtype != torch.int64 or ids.is_cuda or not ids.is_contiguous():
+            raise ValueError("ids must be a contiguous int64 host tensor")
+        removed = ctypes.c_int64(0)
+        _check(load_library().ic_cache_remove(self._h, _ptr(ids), ids.numel(), ctypes.byref(removed)))
+        return int(removed.value)
 
     def set_path(self, path: int) -> None:
         _check(load_library().ic_cache_set_path(self._h, path))

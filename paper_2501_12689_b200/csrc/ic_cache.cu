@@ -83,7 +83,7 @@ struct ic_cache {
   bool own_slab = false;
   int64_t* ids = nullptr;
   bool own_ids = false;
-  Buffer q_bf16, q_f32, partials, thr, pace, stage_in, stage_ids, stage_scores;
+  Buffer q_bf16, q_f32, partials, thr, pace, stage_in, stage_ids, stage_scores, evict;
   unsigned pace_epoch = 0;
   int l2_bytes = 0;
   int* h_status = nullptr;  // pinned, mapped; kernels write a code when a bounded wait expires
@@ -700,6 +700,7 @@ void ic_cache_destroy(ic_cache_t* c) {
   release(c->stage_in);
   release(c->stage_ids);
   release(c->stage_scores);
+  release(c->evict);
   if (c->h_status) cudaFreeHost(c->h_status);
   for (cudaEvent_t ev : c->ev_score) cudaEventDestroy(ev);
   for (cudaEvent_t ev : c->ev_merge) cudaEventDestroy(ev);
@@ -828,6 +829,72 @@ int ic_cache_query_host(ic_cache_t* c, const void* q_host, int32_t nq, int32_t k
   if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
   if (e != cudaSuccess) return fail(IC_ERR_CUDA, "result copy failed: %s", cudaGetErrorString(e));
   return check_timeout(c);
+}
+
+int ic_cache_remove(ic_cache_t* c, const int64_t* ids_host, int64_t n, int64_t* n_removed) {
+  if (n_removed) *n_removed = 0;
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  if (n < 0) return fail(IC_ERR_INVALID, "n %lld < 0", (long long)n);
+  if (n == 0 || c->size == 0) return IC_OK;
+  if (!ids_host) return fail(IC_ERR_INVALID, "NULL pointer with n > 0");
+  DeviceGuard guard(c->device);
+  int rc = check_timeout(c);
+  if (rc != IC_OK) return rc;
+  // the ids to drop, sorted and without repeats
+  std::vector<int64_t> wanted(ids_host, ids_host + n);
+  std::sort(wanted.begin(), wanted.end());
+  wanted.erase(std::unique(wanted.begin(), wanted.end()), wanted.end());
+  const int64_t nw = (int64_t)wanted.size();
+  // device scratch: [wanted nw][count 1][matches cap][src cap][dst cap]
+  const int64_t cap = std::min<int64_t>(c->size, 4 * nw + 1024);
+  const size_t words = (size_t)nw + 1 + 3 * (size_t)cap;
+  if ((rc = ensure(c, c->evict, words * 8, "eviction scratch")) != IC_OK) return rc;
+  int64_t* d_wanted = static_cast<int64_t*>(c->evict.p);
+  unsigned long long* d_count = reinterpret_cast<unsigned long long*>(d_wanted + nw);
+  int64_t* d_match = d_wanted + nw + 1;
+  int64_t* d_src = d_match + cap;
+  int64_t* d_dst = d_src + cap;
+  cudaError_t e = cudaMemcpyAsync(d_wanted, wanted.data(), (size_t)nw * 8, cudaMemcpyHostToDevice, c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(d_count, 0, 8, c->stream);
+  if (e == cudaSuccess) e = icc::launch_find_ids(c->ids, c->size, d_wanted, nw, d_match, d_count, cap, c->stream);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "id search launch failed: %s", cudaGetErrorString(e));
+  c->launches += 1;
+  unsigned long long m = 0;
+  e = cudaMemcpyAsync(&m, d_count, 8, cudaMemcpyDeviceToHost, c->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "id search failed: %s", cudaGetErrorString(e));
+  if (m == 0) return IC_OK;
+  if ((int64_t)m > cap)
+    return fail(IC_ERR_UNSUPPORTED, "%llu entries carry the %lld given ids (more than %lld): remove them in smaller groups",
+                m, (long long)nw, (long long)cap);
+  std::vector<int64_t> gone((size_t)m);
+  e = cudaMemcpy(gone.data(), d_match, (size_t)m * 8, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "match copy failed: %s", cudaGetErrorString(e));
+  std::sort(gone.begin(), gone.end());
+  // vacated slots below the new size are refilled, in order, by the surviving rows of the tail
+  const int64_t new_size = c->size - (int64_t)m;
+  std::vector<int64_t> src, dst;
+  size_t gi = std::lower_bound(gone.begin(), gone.end(), new_size) - gone.begin();   // first removed slot in the tail
+  int64_t tail = new_size;
+  for (size_t h = 0; h < gone.size() && gone[h] < new_size; ++h) {
+    while (gi < gone.size() && gone[gi] == tail) {   // skip tail rows that are removed themselves
+      ++gi;
+      ++tail;
+    }
+    dst.push_back(gone[h]);
+    src.push_back(tail++);
+  }
+  if (!src.empty()) {
+    e = cudaMemcpyAsync(d_src, src.data(), src.size() * 8, cudaMemcpyHostToDevice, c->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d_dst, dst.data(), dst.size() * 8, cudaMemcpyHostToDevice, c->stream);
+    if (e == cudaSuccess) e = icc::launch_move_rows(c->slab, c->ids, d_src, d_dst, (int64_t)src.size(), c->dim, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);   // src/dst are host vectors about to go away
+    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "row move failed: %s", cudaGetErrorString(e));
+    c->launches += 1;
+  }
+  c->size = new_size;
+  if (n_removed) *n_removed = (int64_t)m;
+  return IC_OK;
 }
 
 int ic_cache_set_stream(ic_cache_t* c, void* cuda_stream) {

@@ -41,6 +41,14 @@ cudaError_t launch_convert_rows(const void* in, int in_is_f32, int64_t nrows, in
                                 void* out_bf16, float* out_f32, int64_t pad_rows, const int64_t* ids_in,
                                 int64_t* ids_out, cudaStream_t st);
 
+// Eviction support: slots whose id is in the sorted list `wanted` are appended (any order) to
+// match_slots (capacity cap) and counted in *match_count (which may exceed cap).
+cudaError_t launch_find_ids(const int64_t* ids, int64_t n, const int64_t* wanted, int64_t n_wanted, int64_t* match_slots,
+                            unsigned long long* match_count, int64_t cap, cudaStream_t st);
+// Move rows (and ids) inside the slab, src[i] -> dst[i]; the two sets must be disjoint.
+cudaError_t launch_move_rows(void* slab, int64_t* ids, const int64_t* src, const int64_t* dst, int64_t nmoves, int dim,
+                             cudaStream_t st);
+
 // Generic CUDA-core scoring of up to 4 queries [q0, q0+4) against rows [0, n).
 // partials: [n_part][nq][k] packed keys.
 cudaError_t launch_generic(const void* slab, int64_t n, int dim, const float* q_f32, int q0, int nq,

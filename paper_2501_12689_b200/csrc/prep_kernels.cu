@@ -89,4 +89,60 @@ cudaError_t launch_convert_rows(const void* in, int in_is_f32, int64_t nrows, in
                            normalize, static_cast<__nv_bfloat16*>(out_bf16), out_f32, pad_rows, ids_in, ids_out);
 }
 
+// Eviction support.  find_ids_kernel lists the slots whose id is one of `wanted` (sorted
+// ascending, n_wanted entries): one thread per cache row, binary search, matches appended
+// through an atomic counter (their order is arbitrary; the host sorts them).
+__global__ void __launch_bounds__(256)
+find_ids_kernel(const int64_t* __restrict__ ids, int64_t n, const int64_t* __restrict__ wanted, int64_t n_wanted,
+                int64_t* __restrict__ match_slots, unsigned long long* __restrict__ match_count, int64_t cap) {
+  grid_dep_launch_dependents();
+  grid_dep_wait();
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int64_t id = ids[i];
+  int64_t lo = 0, hi = n_wanted;
+  while (lo < hi) {
+    const int64_t mid = (lo + hi) >> 1;
+    if (wanted[mid] < id) lo = mid + 1;
+    else hi = mid;
+  }
+  if (lo < n_wanted && wanted[lo] == id) {
+    const unsigned long long pos = atomicAdd(match_count, 1ull);
+    if ((int64_t)pos < cap) match_slots[pos] = i;
+  }
+}
+
+// Copy whole rows (and their ids) inside the slab: row src[i] -> row dst[i].  The two sets are
+// disjoint (tail rows move into vacated slots), so rows can move in parallel.
+__global__ void __launch_bounds__(CONV_WARPS * 32)
+move_rows_kernel(__nv_bfloat16* __restrict__ slab, int64_t* __restrict__ ids, const int64_t* __restrict__ src,
+                 const int64_t* __restrict__ dst, int64_t nmoves, int dim) {
+  grid_dep_launch_dependents();
+  grid_dep_wait();
+  const int lane = threadIdx.x & 31;
+  const int64_t i = (int64_t)blockIdx.x * CONV_WARPS + (threadIdx.x >> 5);
+  if (i >= nmoves) return;
+  const int64_t s = src[i], d = dst[i];
+  const uint4* from = reinterpret_cast<const uint4*>(slab + s * dim);
+  uint4* to = reinterpret_cast<uint4*>(slab + d * dim);
+  for (int c = lane; c < (dim >> 3); c += 32) to[c] = from[c];
+  if (lane == 0) ids[d] = ids[s];
+}
+
+cudaError_t launch_find_ids(const int64_t* ids, int64_t n, const int64_t* wanted, int64_t n_wanted, int64_t* match_slots,
+                            unsigned long long* match_count, int64_t cap, cudaStream_t st) {
+  if (n == 0 || n_wanted == 0) return cudaSuccess;
+  const unsigned blocks = (unsigned)((n + 255) / 256);
+  return launch_overlapped(find_ids_kernel, dim3(blocks), dim3(256), 0, st, 1, ids, n, wanted, n_wanted, match_slots,
+                           match_count, cap);
+}
+
+cudaError_t launch_move_rows(void* slab, int64_t* ids, const int64_t* src, const int64_t* dst, int64_t nmoves, int dim,
+                             cudaStream_t st) {
+  if (nmoves == 0) return cudaSuccess;
+  const unsigned blocks = (unsigned)((nmoves + CONV_WARPS - 1) / CONV_WARPS);
+  return launch_overlapped(move_rows_kernel, dim3(blocks), dim3(CONV_WARPS * 32), 0, st, 1,
+                           static_cast<__nv_bfloat16*>(slab), ids, src, dst, nmoves, dim);
+}
+
 }  // namespace icc

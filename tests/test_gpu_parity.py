@@ -268,3 +268,49 @@ def test_min_score_filter_and_counts(path):
     with ICCache(w.dim, 10) as c:
         with pytest.raises(ICCacheError):
             c.query_min_score(q, 3, float("nan"))
+
+
+@pytest.mark.parametrize("path", ["scan", "umma"])
+def test_remove_closes_gaps_and_frees_capacity(path):
+    n, dim, k = 30_000, 128, 12
+    nq = 2 if path == "scan" else 33
+    x, q = _gauss(n, dim, nq, seed=120)
+    lab = wl.labels(n, DEV)
+    g = torch.Generator().manual_seed(121)
+    with ICCache(dim, n) as c:
+        c.set_path(PATHS[path])
+        c.insert(x, lab)
+        # victims: the best match of every query, the first and last rows, a random 10 %, an id
+        # that does not exist and a repeated id
+        ids0, _ = c.query(q, 1)
+        victims = torch.cat([ids0.flatten().cpu(), lab[:3].cpu(), lab[-5:].cpu(),
+                             lab.cpu()[torch.randperm(n, generator=g)[: n // 10]],
+                             torch.tensor([12345, int(lab[7])])])
+        removed = c.remove(victims.contiguous())
+        keep = ~torch.isin(lab.cpu(), victims)
+        assert removed == int((~keep).sum()) and c.size == int(keep.sum())
+        xr, lr = x.cpu()[keep], lab.cpu()[keep]
+
+        def check(rows, labels, what):
+            ids, sc = c.query(q, k)
+            c.sync()
+            ref = oracle.search(wl.as_bits(rows), wl.as_bits(q), k, ids=labels.numpy(), want_all_scores=True)
+            oracle.accept(ids.cpu().numpy(), sc.cpu().numpy(), ref["all_scores"], k, ids=labels.numpy(), tol=1e-4, what=what)
+            return ids
+        ids1 = check(xr, lr, f"after remove/{path}")
+        assert not torch.isin(ids1.cpu(), victims).any()
+        # the freed capacity takes new rows
+        extra = wl.queries(wl.Workload("g", n, dim, "bf16", (1,), 8, seed=122), removed, DEV)
+        extra_lab = wl.labels(removed, DEV, first_slot=n)
+        c.insert(extra, extra_lab)
+        assert c.size == n
+        check(torch.cat([xr, extra.cpu()]), torch.cat([lr, extra_lab.cpu()]), f"after refill/{path}")
+        with pytest.raises(ICCacheError):
+            c.insert(extra[:1], extra_lab[:1])
+        # removing ids that are not there changes nothing; removing everything empties the cache
+        assert c.remove(torch.tensor([1, 2, 3])) == 0 and c.size == n
+        everything = torch.cat([lr, extra_lab.cpu()])
+        assert c.remove(everything) == n and c.size == 0
+        ids, sc = c.query(q, 3)
+        c.sync()
+        assert torch.all(ids == -1)
