@@ -205,11 +205,16 @@ int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32
     const char* seed_env = getenv("IC_CACHE_SEED");   // tuning knob: "0" scores everything in one pass
     const bool seeding = !(seed_env && seed_env[0] == '0' && seed_env[1] == 0);
     if (seeding && n_tiles >= (int64_t)SEED_MIN_TILES_PER_CTA * out->n_partitions) {
-      const int64_t t = n_tiles / SEED_FRACTION / out->n_partitions * out->n_partitions;
+      int seed_fraction = SEED_FRACTION;
+      if (const char* fe = getenv("IC_CACHE_SEED_FRACTION")) {   // tuning knob: 1/fraction of the tiles are sampled
+        const int f = atoi(fe);
+        if (f >= 2) seed_fraction = f;
+      }
+      const int64_t t = n_tiles / seed_fraction / out->n_partitions * out->n_partitions;
       out->seed_tiles = (int32_t)std::max<int64_t>(out->n_partitions, t);
       // with several tiles per CTA in that sample, seed the sample itself from one tile per CTA
       if (out->seed_tiles >= SEED_TWO_LEVEL_TILES_PER_CTA * out->n_partitions)
-        out->seed0_tiles = std::max(out->n_partitions, out->seed_tiles / SEED_FRACTION / out->n_partitions * out->n_partitions);
+        out->seed0_tiles = std::max(out->n_partitions, out->seed_tiles / 16 / out->n_partitions * out->n_partitions);
     }
     // 1 KiB alignment slack + 256 B of barriers, the per-query lists, then as many candidate
     // queue entries per query (up to 8) as still leave room for two ring stages

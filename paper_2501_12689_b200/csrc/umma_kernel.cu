@@ -367,14 +367,42 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           const float best = fmaxf(fmaxf(fmaxf(g[0], g[1]), fmaxf(g[2], g[3])), fmaxf(fmaxf(g[4], g[5]), fmaxf(g[6], g[7])));
           active = __any_sync(FULL_MASK, best >= thr_score);   // common case: nothing passes
         }
-        // Everything below is warp-uniform control flow, and the queue is drained at one place
-        // only (the code stays small and a drain is always entered by all 32 lanes, each working
-        // through its own queue).  Columns are considered in order; whenever some lane's queue
-        // could not take another group of four (or, for queues shorter than four, another
-        // entry) the pass stops, the queues are drained and the pass resumes at c_next.
+        // Common slow case: every lane's queue has room for all of its passing columns.  One
+        // vote establishes that, one OR-reduction tells which groups of columns anybody needs,
+        // and the pushes are predicated stores: no per-group votes, no divergent branches.
+        bool drain_after = false;
+        if (active) {
+          uint32_t hm = 0;
+#pragma unroll
+          for (int c = 0; c < 32; ++c) hm |= (__uint_as_float(v[c]) >= thr_score) ? (1u << c) : 0u;
+          if (!__any_sync(FULL_MASK, cnt + __popc(hm) > qcap)) {
+            const uint32_t cols = __reduce_or_sync(FULL_MASK, hm);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              if ((cols >> (4 * j)) & 0xfu) {   // warp-uniform
+#pragma unroll
+                for (int c = 4 * j; c < 4 * j + 4; ++c) {
+                  if ((hm >> c) & 1u) {
+                    my_queue[cnt * 32] = ((uint64_t)v[c] << 32) | (uint32_t)(col0 + c);
+                    ++cnt;
+                  }
+                }
+              }
+            }
+            active = false;
+            drain_after = __any_sync(FULL_MASK, 2 * cnt >= qcap);
+          }
+        }
+        // Otherwise (cold start, very loose thresholds): warp-uniform control flow with the queue
+        // drained at one place only (the code stays small and a drain is always entered by all
+        // 32 lanes, each working through its own queue).  Columns are considered in order;
+        // whenever some lane's queue could not take another group of four (or, for queues
+        // shorter than four, another entry) the pass stops, the queues are drained and the pass
+        // resumes at c_next.
         int c_next = 0;
         while (true) {
-          bool need_drain = false;
+          bool need_drain = drain_after;
+          drain_after = false;
           if (active) {
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
