@@ -8,5 +8,6 @@ from .ic_oracle import (  # noqa: F401
     bf16_bits_to_f32,
     f32_to_bf16_bits,
     search,
+    self_similarity,
 )
 from .check import accept, AcceptanceError  # noqa: F401

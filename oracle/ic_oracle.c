@@ -181,3 +181,35 @@ void ic_oracle_apply_min_score(int64_t* out_ids, float* out_scores, int64_t* out
     if (counts) counts[iq] = kept;
   }
 }
+
+/*
+ * Top-1 similarity of cached entries to the OTHER cached entries (the request-similarity
+ * study of paper Sec. 2.2: "top-1 request similarities of each request to others").
+ * For every row i in [first, first+count): the row j != i with the largest fp32 dot product
+ * (ties: lowest slot).  out_ids/out_slots/out_scores have `count` entries; with fewer than two
+ * rows in the cache the answer is (-1, -1, -inf).  Plain double loop, no blocking.
+ */
+int ic_oracle_self_similarity(const void* X, int x_dtype, const int64_t* ids, int64_t n, int32_t d, int64_t first,
+                              int64_t count, int threads, int64_t* out_ids, float* out_scores, int64_t* out_slots) {
+  if (n < 0 || d <= 0 || first < 0 || count < 0 || first + count > n) return -1;
+  if (threads < 1) threads = 1;
+#pragma omp parallel for num_threads(threads) schedule(static)
+  for (int64_t r = 0; r < count; ++r) {
+    const int64_t i = first + r;
+    float best = -INFINITY;
+    int64_t best_j = -1;
+    for (int64_t j = 0; j < n; ++j) {
+      if (j == i) continue;
+      float acc = 0.0f;
+      for (int32_t t = 0; t < d; ++t) acc += load_elem(X, x_dtype, i * (int64_t)d + t, 0) * load_elem(X, x_dtype, j * (int64_t)d + t, 0);
+      if (best_j < 0 || acc > best) {
+        best = acc;
+        best_j = j;
+      }
+    }
+    out_scores[r] = best;
+    if (out_slots) out_slots[r] = best_j;
+    if (out_ids) out_ids[r] = best_j < 0 ? -1 : (ids ? ids[best_j] : best_j);
+  }
+  return 0;
+}

@@ -61,6 +61,10 @@ def _load():
         lib.ic_oracle_apply_min_score.restype = None
         lib.ic_oracle_apply_min_score.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32,
                                                   ctypes.c_int32, ctypes.c_float, ctypes.c_void_p]
+        lib.ic_oracle_self_similarity.restype = ctypes.c_int
+        lib.ic_oracle_self_similarity.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_int64,
+                                                  ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, ctypes.c_int,
+                                                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -150,3 +154,23 @@ def search(x, q, k: int, ids=None, normalize: bool = False, round_bf16: bool = F
                                       float(min_score), counts.ctypes.data)
         res["counts"] = counts
     return res
+
+
+def self_similarity(x, first: int = 0, count: int | None = None, ids=None, threads: int | None = None):
+    """For rows first .. first+count-1 of x: the most similar OTHER row (fp32 dot product, ties to
+    the lower slot).  Returns dict(ids, scores, slots), each of length count."""
+    lib = _load()
+    x, xdt = _as_matrix(x, "x")
+    n, d = x.shape
+    count = n - first if count is None else count
+    if ids is not None:
+        ids = np.ascontiguousarray(ids, dtype=np.int64)
+    out_ids = np.empty((count,), dtype=np.int64)
+    out_scores = np.empty((count,), dtype=np.float32)
+    out_slots = np.empty((count,), dtype=np.int64)
+    rc = lib.ic_oracle_self_similarity(x.ctypes.data, xdt, ids.ctypes.data if ids is not None else None, n, d,
+                                       first, count, int(threads or default_threads()), out_ids.ctypes.data,
+                                       out_scores.ctypes.data, out_slots.ctypes.data)
+    if rc != 0:
+        raise RuntimeError(f"ic_oracle_self_similarity failed with code {rc}")
+    return {"ids": out_ids, "scores": out_scores, "slots": out_slots}

@@ -29,6 +29,8 @@ def _parse_golden():
         elif tok[0] == "x":
             assert int(tok[1]) == len(cur["x"])
             cur["x"].append([float(v) for v in tok[2:]])
+        elif tok[0] == "self":
+            caches[tok[1]].setdefault("self", {})[int(tok[2])] = (int(tok[4].split(":")[0]), float(tok[4].split(":")[1]))
         elif tok[0] == "q":
             arrow = tok.index("->")
             vec = [float(v) for v in tok[1:arrow]]
@@ -316,3 +318,24 @@ def test_min_score_filter_hand_computed():
     assert oracle.search(x, q[:1], k=5, min_score=1.0)["counts"].tolist() == [1]
     assert oracle.search(x, q[:1], k=5, min_score=1.5)["counts"].tolist() == [0]
     assert oracle.search(x, q[:1], k=7, min_score=-np.inf)["counts"].tolist() == [5]
+
+
+# ---------------------------------------------------------------- similarity to the other entries
+
+def test_self_similarity_hand_computed_and_against_search():
+    c = _parse_golden()["axes"]
+    x = np.array(c["x"], dtype=np.float32)
+    r = oracle.self_similarity(x)
+    assert r["slots"].tolist() == [c["self"][i][0] for i in range(5)]
+    np.testing.assert_allclose(r["scores"], [c["self"][i][1] for i in range(5)], atol=1e-6)
+    # a row's best other row is the first entry of its own top-2 that is not the row itself
+    xs, _ = _tiny(n=700, d=48)
+    xs[13] = xs[400]                      # an exact duplicate pair: each is the other's best
+    full = oracle.search(xs, xs, k=2)
+    want = [row[0] if row[0] != i else row[1] for i, row in enumerate(full["slots"])]
+    got = oracle.self_similarity(xs, threads=3)
+    assert got["slots"].tolist() == want and got["slots"][13] == 400 and got["slots"][400] == 13
+    part = oracle.self_similarity(xs, first=100, count=50, ids=np.arange(700, dtype=np.int64) + 7)
+    assert part["ids"].tolist() == [w + 7 for w in want[100:150]]
+    one = oracle.self_similarity(xs[:1])
+    assert one["slots"].tolist() == [-1] and np.isneginf(one["scores"][0])
