@@ -52,6 +52,8 @@ def parse_args():
     ap.add_argument("--no-sweep", action="store_true", help="skip the secondary batch sizes")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--self-similarity-rows", type=int, default=0,
+                    help="also time the all-pairs top-1 self-similarity over this many cached rows")
     return ap.parse_args()
 
 
@@ -267,6 +269,21 @@ def run_ours(args):
             if q != nq:
                 sweep.append(measure(q, min(steps, 200), max(3, min(warmup, 5)), profiled=True))
 
+    self_sim = None
+    if args.self_similarity_rows > 0:
+        rows = min(args.self_similarity_rows, cache.size)
+        cache.self_similarity(0, min(rows, 2048))            # warm-up (grows scratch)
+        cache.sync()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_now = cache.size
+        ev0.record()
+        cache.self_similarity(0, rows)
+        ev1.record()
+        torch.cuda.synchronize()
+        ms = ev0.elapsed_time(ev1)
+        self_sim = {"rows": rows, "cache_rows": n_now, "ms": ms, "rows_per_sec": rows / (ms * 1e-3),
+                    "tflops": 2.0 * rows * n_now * w.dim / (ms * 1e-3) / 1e12}
+
     clocks = sampler.stop() if sampler else None
 
     ms_all, q_all = aggregate_ranks(dist, main["ms"], float(nq * steps))
@@ -343,6 +360,7 @@ def run_ours(args):
         "roofline": roof,
         "profiled_region": {"ms_per_step": prof["ms"] / steps},
         "clocks": clocks,
+        "self_similarity": self_sim,
         "sweep": [{"nq": r["nq"], "queries_per_sec": r["nq"] * r["steps"] / (r["ms"] * 1e-3),
                    "ms_per_step": r["ms"] / r["steps"], "roofline": roofline_of(r)} for r in sweep],
     }

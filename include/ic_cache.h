@@ -185,6 +185,19 @@ int ic_cache_query_static(ic_cache_t* c, const void* q, int32_t nq, int32_t k, i
 int ic_cache_insert_host(ic_cache_t* c, const void* emb_host, const int64_t* ids_host, int64_t n);
 
 /*
+ * Similarity of cached entries to the OTHER cached entries (the request-similarity study of
+ * paper Sec. 2.2: top-1 similarity of each request to the others).  For each of the `count`
+ * entries in slots [first, first+count): the id and score of the best-scoring entry other than
+ * itself (an exact copy of it counts as another entry; ties go to the lower slot).
+ * out_ids [count] int64, out_scores [count] fp32, device pointers; (-1, -infinity) when the
+ * cache holds a single entry.  The stored bf16 rows serve as the queries; work is
+ * count * size * dim multiply-adds on the tensor-core path, in passes of 1024 entries.
+ * Stream-ordered like ic_cache_query; may grow scratch on first use.
+ */
+int ic_cache_self_similarity(ic_cache_t* c, int64_t first, int64_t count, int64_t* out_ids,
+                             float* out_scores);
+
+/*
  * Eviction mechanics (paper Sec. 4.3, "Example Manager": a background solver picks the
  * examples to drop when the cache is full; which ones is the caller's policy).  Removes every
  * entry whose id equals one of ids_host[0..n) (HOST array; ids that match nothing are

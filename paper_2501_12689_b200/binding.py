@@ -69,6 +69,8 @@ SIGNATURES = {
     "ic_cache_query_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
                                            ctypes.c_void_p, ctypes.c_void_p]),
     "ic_cache_insert_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64]),
+    "ic_cache_self_similarity": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
+                                                ctypes.c_void_p]),
     "ic_cache_remove": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.POINTER(ctypes.c_int64)]),
     "ic_cache_destroy": (None, [ctypes.c_void_p]),
     "ic_cache_set_stream": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
@@ -282,6 +284,14 @@ class ICCache:
         if out_scores is None:
             out_scores = torch.empty(nq, k, dtype=torch.float32).pin_memory()
         ic_cache_query_host(self._h, q, nq, k, out_ids, out_scores)
+        return out_ids, out_scores
+
+    def self_similarity(self, first: int = 0, count: Optional[int] = None):
+        """Best other entry (id, score) for the entries in slots [first, first+count)."""
+        count = self.size - first if count is None else count
+        out_ids = torch.empty(count, dtype=torch.int64, device=self.device)
+        out_scores = torch.empty(count, dtype=torch.float32, device=self.device)
+        _check(load_library().ic_cache_self_similarity(self._h, first, count, _ptr(out_ids), _ptr(out_scores)))
         return out_ids, out_scores
 
     def remove(self, ids: torch.Tensor) -> int:

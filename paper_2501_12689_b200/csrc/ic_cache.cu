@@ -902,6 +902,44 @@ int ic_cache_remove(ic_cache_t* c, const int64_t* ids_host, int64_t n, int64_t* 
   return IC_OK;
 }
 
+int ic_cache_self_similarity(ic_cache_t* c, int64_t first, int64_t count, int64_t* out_ids, float* out_scores) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  if (first < 0 || count < 0 || first + count > c->size)
+    return fail(IC_ERR_INVALID, "rows [%lld, %lld) are not all cached (size %lld)", (long long)first, (long long)(first + count), (long long)c->size);
+  if (count == 0) return IC_OK;
+  if (!out_ids || !out_scores) return fail(IC_ERR_INVALID, "NULL pointer with count > 0");
+  DeviceGuard guard(c->device);
+  if (!is_device_ptr(out_ids, c->device) || !is_device_ptr(out_scores, c->device))
+    return fail(IC_ERR_INVALID, "out_ids and out_scores must be device pointers on device %d", c->device);
+  int rc = check_timeout(c);
+  if (rc != IC_OK) return rc;
+  const int k = 2;   // a row's best match is itself or an exact copy; the next one is the answer
+  for (int64_t w0 = 0; w0 < count; w0 += WINDOW_MAX_NQ) {
+    const int nq = (int)std::min<int64_t>(WINDOW_MAX_NQ, count - w0);
+    ic_cache_plan_t pl;
+    if ((rc = plan_impl(c->dim, c->size, nq, k, IC_PATH_UMMA, c->sm_count, c->smem_optin, &pl)) != IC_OK) return rc;
+    const size_t list_block = (size_t)nq * k;
+    if ((rc = ensure(c, c->partials, (size_t)(2 * pl.n_partitions + 2) * list_block * 8, "partial top-k lists")) != IC_OK) return rc;
+    if ((rc = ensure(c, c->thr, (size_t)nq * 8, "seed thresholds")) != IC_OK) return rc;
+    uint64_t* partials = static_cast<uint64_t*>(c->partials.p);
+    int n_final_lists = 0;
+    // the queries are the stored bf16 rows themselves: the query tensor map points into the slab
+    // (rows past nq read as zero), no conversion pass is needed
+    const char* q_rows = static_cast<const char*>(c->slab) + (size_t)(first + w0) * c->dim * 2;
+    // (the map may cover following slab rows up to a full 128-row tile, never past the slab;
+    // lanes beyond nq are not real queries, whatever they read)
+    const int q_map_rows = (int)std::min<int64_t>((nq + QUERY_TILE - 1) / QUERY_TILE * QUERY_TILE, c->capacity - (first + w0));
+    rc = run_umma_passes(c, pl, q_rows, nq, q_map_rows, k, partials, static_cast<uint64_t*>(c->thr.p),
+                         static_cast<unsigned long long*>(c->pace.p), &n_final_lists, false);
+    if (rc != IC_OK) return rc;
+    cudaError_t e = icc::launch_merge(partials, n_final_lists, nq, k, c->ids, out_ids + w0, out_scores + w0, -INFINITY,
+                                      nullptr, c->stream, first + w0);
+    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "merge launch failed: %s", cudaGetErrorString(e));
+    c->launches += 1;
+  }
+  return IC_OK;
+}
+
 int ic_cache_set_stream(ic_cache_t* c, void* cuda_stream) {
   if (!c) return fail(IC_ERR_INVALID, "NULL handle");
   c->stream = static_cast<cudaStream_t>(cuda_stream);

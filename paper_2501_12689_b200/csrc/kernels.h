@@ -102,7 +102,9 @@ cudaError_t umma_configure(int smem_optin);
 // receives the number of entries kept per query.
 cudaError_t launch_merge(const uint64_t* partials, int n_part, int nq, int k, const int64_t* ids,
                          int64_t* out_ids, float* out_scores, float min_score, int32_t* out_counts,
-                         cudaStream_t st);
+                         cudaStream_t st, int64_t self_slot0 = -1);
+// self_slot0 >= 0: query q is cache row self_slot0 + q; out_ids/out_scores then hold ONE entry
+// per query, the best-scoring entry other than that row.
 // Same merge, but the result stays in key form: out_keys [nq][k] (sorted, KEY_EMPTY padded)
 // and out_thr [nq] = the k-th key (KEY_EMPTY when fewer than k candidates exist).
 cudaError_t launch_merge_keys(const uint64_t* partials, int n_part, int nq, int k, uint64_t* out_keys,

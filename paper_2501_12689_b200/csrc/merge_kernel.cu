@@ -47,7 +47,8 @@ __global__ void __launch_bounds__(MERGE_THREADS)
 merge_topk_kernel(const uint64_t* __restrict__ partials, int n_part, int nq, int k,
                   const int64_t* __restrict__ ids, int64_t* __restrict__ out_ids,
                   float* __restrict__ out_scores, uint64_t* __restrict__ out_keys,
-                  uint64_t* __restrict__ out_thr, float min_score, int32_t* __restrict__ out_counts) {
+                  uint64_t* __restrict__ out_thr, float min_score, int32_t* __restrict__ out_counts,
+                  int64_t self_slot0) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint64_t* cand = reinterpret_cast<uint64_t*>(smem_raw);                 // [n_part][k]
   uint32_t* pos = reinterpret_cast<uint32_t*>(cand + (size_t)n_part * k);  // [n_part]
@@ -81,6 +82,23 @@ merge_topk_kernel(const uint64_t* __restrict__ partials, int n_part, int nq, int
   if (out_keys) {  // intermediate merge: keep the key form
     for (int i = tid; i < k; i += MERGE_THREADS) out_keys[(size_t)q * k + i] = win_key[i];
     if (tid == 0) out_thr[q] = win_key[k - 1];
+    return;
+  }
+  if (self_slot0 >= 0) {
+    // similarity to the OTHER entries: query q is cache row self_slot0 + q; report the best
+    // entry that is not that row (one result per query)
+    if (tid == 0) {
+      uint64_t pick = KEY_EMPTY;
+      for (int i = 0; i < k; ++i) {
+        const uint64_t key = win_key[i];
+        if (key != KEY_EMPTY && (int64_t)key_slot(key) != self_slot0 + q) {
+          pick = key;
+          break;
+        }
+      }
+      out_scores[q] = (pick == KEY_EMPTY) ? -INFINITY : key_score(pick);
+      out_ids[q] = (pick == KEY_EMPTY) ? (int64_t)-1 : ids[key_slot(pick)];
+    }
     return;
   }
   // Entries below min_score (-inf = keep all) are reported as absent; the list is sorted, so
@@ -117,11 +135,12 @@ cudaError_t merge_configure(int smem_optin) {
 
 cudaError_t launch_merge(const uint64_t* partials, int n_part, int nq, int k, const int64_t* ids,
                          int64_t* out_ids, float* out_scores, float min_score, int32_t* out_counts,
-                         cudaStream_t st) {
+                         cudaStream_t st, int64_t self_slot0) {
   const size_t smem = (size_t)n_part * k * 8 + (size_t)n_part * 4;
   if (smem > (size_t)g_merge_smem_limit) return cudaErrorInvalidValue;
   return launch_overlapped(merge_topk_kernel, dim3(nq), dim3(MERGE_THREADS), smem, st, 1, partials, n_part, nq, k, ids,
-                           out_ids, out_scores, (uint64_t*)nullptr, (uint64_t*)nullptr, min_score, out_counts);
+                           out_ids, out_scores, (uint64_t*)nullptr, (uint64_t*)nullptr, min_score, out_counts,
+                           self_slot0);
 }
 
 cudaError_t launch_merge_keys(const uint64_t* partials, int n_part, int nq, int k, uint64_t* out_keys,
@@ -130,7 +149,7 @@ cudaError_t launch_merge_keys(const uint64_t* partials, int n_part, int nq, int 
   if (smem > (size_t)g_merge_smem_limit || !out_keys || !out_thr) return cudaErrorInvalidValue;
   return launch_overlapped(merge_topk_kernel, dim3(nq), dim3(MERGE_THREADS), smem, st, 1, partials, n_part, nq, k,
                            (const int64_t*)nullptr, (int64_t*)nullptr, (float*)nullptr, out_keys, out_thr, -INFINITY,
-                           (int32_t*)nullptr);
+                           (int32_t*)nullptr, (int64_t)-1);
 }
 
 }  // namespace icc

@@ -314,3 +314,39 @@ def test_remove_closes_gaps_and_frees_capacity(path):
         ids, sc = c.query(q, 3)
         c.sync()
         assert torch.all(ids == -1)
+
+
+@pytest.mark.parametrize("n,dim", [(5, 64), (1, 64), (6_000, 128), (2_500, 768)])
+def test_self_similarity_matches_oracle(n, dim):
+    x, _ = _gauss(n, dim, 1, seed=130 + n)
+    if n > 100:
+        x[17] = x[n - 3]                       # an exact duplicate pair: each is the other's best
+        x[40] = x[41] = x[42]                  # a triple
+    lab = wl.labels(n, DEV)
+    with ICCache(dim, n) as c:
+        c.insert(x, lab)
+        ids, sc = c.self_similarity()
+        c.sync()
+        ref = oracle.self_similarity(wl.as_bits(x), ids=lab.cpu().numpy())
+        got_ids, got_sc = ids.cpu().numpy(), sc.cpu().numpy()
+        if n == 1:
+            assert got_ids.tolist() == [-1] and np.isneginf(got_sc[0])
+            return
+        assert np.allclose(got_sc, ref["scores"], atol=1e-4)
+        # the partner may differ only where two candidates score within rounding distance
+        differ = np.flatnonzero(got_ids != ref["ids"])
+        xb = x.float().cpu()
+        labc = lab.cpu().numpy()
+        for i in differ:
+            j = int(np.flatnonzero(labc == got_ids[i])[0])
+            assert j != i and abs(float(xb[i] @ xb[j]) - float(ref["scores"][i])) < 1e-4
+        assert differ.size <= max(2, n // 200)
+        if n > 100:
+            assert got_ids[17] == labc[n - 3] and got_ids[n - 3] == labc[17] and abs(got_sc[17] - 1.0) < 5e-3
+            assert got_ids[40] == labc[41] and got_ids[41] == labc[40] and got_ids[42] == labc[40]
+        # a sub-range gives the same answers
+        ids2, sc2 = c.self_similarity(first=n // 2, count=min(n - n // 2, 1500))
+        c.sync()
+        assert torch.equal(ids2, ids[n // 2: n // 2 + ids2.numel()])
+        with pytest.raises(ICCacheError):
+            c.self_similarity(first=n - 1, count=5)
