@@ -232,6 +232,16 @@ int ic_cache_clear(ic_cache_t* c);
  * call of this function gave up on a bounded wait, IC_ERR_CUDA on a CUDA error, else IC_OK. */
 int ic_cache_sync(ic_cache_t* c);
 
+/*
+ * Diagnostic for the failure path.  Every device-side wait in this library is bounded; this
+ * call enqueues a one-thread kernel whose wait is made to run out after about a millisecond
+ * (it waits for a barrier that nothing completes) and which then reports the expiry the way a
+ * scoring kernel would.  Afterwards ic_cache_query / ic_cache_insert return IC_ERR_TIMEOUT
+ * until ic_cache_sync has reported and cleared it; the cache contents are untouched and the
+ * handle stays usable.  Lets a caller test its "serve without examples" bypass.
+ */
+int ic_cache_probe_wait_limit(ic_cache_t* c);
+
 /* Kernels launched by this handle so far (insert, query preparation, scoring, merge). */
 int64_t ic_cache_launch_count(const ic_cache_t* c);
 

@@ -78,6 +78,7 @@ SIGNATURES = {
     "ic_cache_size": (ctypes.c_int64, [ctypes.c_void_p]),
     "ic_cache_clear": (ctypes.c_int, [ctypes.c_void_p]),
     "ic_cache_sync": (ctypes.c_int, [ctypes.c_void_p]),
+    "ic_cache_probe_wait_limit": (ctypes.c_int, [ctypes.c_void_p]),
     "ic_cache_launch_count": (ctypes.c_int64, [ctypes.c_void_p]),
     "ic_cache_set_profiling": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32]),
     "ic_cache_read_profile": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_double),
@@ -307,6 +308,10 @@ class ICCache:
 
     def set_stream(self, stream: torch.cuda.Stream) -> None:
         _check(load_library().ic_cache_set_stream(self._h, ctypes.c_void_p(stream.cuda_stream)))
+
+    def probe_wait_limit(self) -> None:
+        """Enqueue the diagnostic kernel whose bounded wait expires (see ic_cache_probe_wait_limit)."""
+        _check(load_library().ic_cache_probe_wait_limit(self._h))
 
     def clear(self) -> None:
         _check(load_library().ic_cache_clear(self._h))

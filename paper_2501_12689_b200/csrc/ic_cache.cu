@@ -940,6 +940,15 @@ int ic_cache_self_similarity(ic_cache_t* c, int64_t first, int64_t count, int64_
   return IC_OK;
 }
 
+int ic_cache_probe_wait_limit(ic_cache_t* c) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  DeviceGuard guard(c->device);
+  cudaError_t e = icc::launch_wait_limit_probe(2000000ll /* about a millisecond */, c->d_status, c->stream);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "probe launch failed: %s", cudaGetErrorString(e));
+  c->launches += 1;
+  return IC_OK;
+}
+
 int ic_cache_set_stream(ic_cache_t* c, void* cuda_stream) {
   if (!c) return fail(IC_ERR_INVALID, "NULL handle");
   c->stream = static_cast<cudaStream_t>(cuda_stream);

@@ -49,6 +49,10 @@ cudaError_t launch_find_ids(const int64_t* ids, int64_t n, const int64_t* wanted
 cudaError_t launch_move_rows(void* slab, int64_t* ids, const int64_t* src, const int64_t* dst, int64_t nmoves, int dim,
                              cudaStream_t st);
 
+// Diagnostic: a bounded wait that is made to run out after limit_cycles (nothing completes the
+// barrier); the kernel reports DEV_TIMEOUT_MBAR in the status word and returns.
+cudaError_t launch_wait_limit_probe(long long limit_cycles, int* dev_status, cudaStream_t st);
+
 // Generic CUDA-core scoring of up to 4 queries [q0, q0+4) against rows [0, n).
 // partials: [n_part][nq][k] packed keys.
 cudaError_t launch_generic(const void* slab, int64_t n, int dim, const float* q_f32, int q0, int nq,

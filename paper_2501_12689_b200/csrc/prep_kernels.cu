@@ -145,4 +145,22 @@ cudaError_t launch_move_rows(void* slab, int64_t* ids, const int64_t* src, const
                            static_cast<__nv_bfloat16*>(slab), ids, src, dst, nmoves, dim);
 }
 
+// Exercise of the bounded-wait path: one thread waits, with a short limit, on an mbarrier that
+// nothing ever completes, then reports the expiry exactly as the scoring kernels would.
+__global__ void wait_limit_probe_kernel(long long limit_cycles, int* dev_status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    mbar_fence_init();
+    if (!mbar_wait(&bar, 0, &abort_flag, limit_cycles)) report_status(dev_status, DEV_TIMEOUT_MBAR);
+  }
+}
+
+cudaError_t launch_wait_limit_probe(long long limit_cycles, int* dev_status, cudaStream_t st) {
+  wait_limit_probe_kernel<<<1, 32, 0, st>>>(limit_cycles, dev_status);
+  return cudaGetLastError();
+}
+
 }  // namespace icc

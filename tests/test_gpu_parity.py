@@ -350,3 +350,29 @@ def test_self_similarity_matches_oracle(n, dim):
         assert torch.equal(ids2, ids[n // 2: n // 2 + ids2.numel()])
         with pytest.raises(ICCacheError):
             c.self_similarity(first=n - 1, count=5)
+
+
+def test_expired_device_wait_is_reported_and_the_handle_recovers():
+    # failure detection without a fault: a bounded wait runs out (nothing completes the barrier),
+    # the kernel reports it, the host surfaces IC_ERR_TIMEOUT, and the cache keeps working
+    from paper_2501_12689_b200 import IC_ERR_TIMEOUT
+    x, q = _gauss(5_000, 64, 3, seed=140)
+    with ICCache(64, 5_010) as c:
+        c.insert(x, wl.labels(5_000, DEV))
+        before = c.query(q, 4)
+        c.sync()
+        c.probe_wait_limit()
+        torch.cuda.synchronize()
+        with pytest.raises(ICCacheError) as e:      # the bypass signal: serve without examples
+            c.query(q, 4)
+        assert e.value.status == IC_ERR_TIMEOUT
+        with pytest.raises(ICCacheError) as e:
+            c.insert(x[:1], wl.labels(1, DEV))
+        assert e.value.status == IC_ERR_TIMEOUT and c.size == 5_000
+        with pytest.raises(ICCacheError) as e:      # sync reports it once and clears it
+            c.sync()
+        assert e.value.status == IC_ERR_TIMEOUT
+        c.sync()
+        after = c.query(q, 4)
+        c.sync()
+        assert torch.equal(before[0], after[0]) and torch.equal(before[1], after[1])
