@@ -181,7 +181,12 @@ int ic_cache_query_host(ic_cache_t* c, const void* q_host, int32_t nq, int32_t k
 int ic_cache_query_static(ic_cache_t* c, const void* q, int32_t nq, int32_t k, int64_t* out_ids,
                           float* out_scores);
 
-/* ic_cache_insert for HOST buffers; synchronises the stream before returning. */
+/*
+ * ic_cache_insert for HOST buffers: copies rows and ids to the device (in slices of at most
+ * 64 MiB) and enqueues the insert.  Returns once everything is enqueued; pageable buffers may be
+ * reused at once, PINNED buffers must stay unchanged until a synchronising call
+ * (ic_cache_query_host, ic_cache_sync) has returned.
+ */
 int ic_cache_insert_host(ic_cache_t* c, const void* emb_host, const int64_t* ids_host, int64_t n);
 
 /*

@@ -765,10 +765,9 @@ int ic_cache_insert_host(ic_cache_t* c, const void* emb_host, const int64_t* ids
       return fail(IC_ERR_CUDA, "stream sync failed during host insert");
     }
   }
-  if (cudaStreamSynchronize(c->stream) != cudaSuccess) {
-    c->size = size_before;
-    return fail(IC_ERR_CUDA, "stream sync failed after host insert");
-  }
+  // No final synchronisation: the device staging buffer is only reused by work enqueued later
+  // on the same stream, and pageable host memory has been copied out by the time
+  // cudaMemcpyAsync returns; pinned host buffers must stay untouched until a synchronising call.
   return IC_OK;
 }
 
