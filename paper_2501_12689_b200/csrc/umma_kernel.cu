@@ -266,12 +266,41 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       my_list[pos * 32] = key;
       return root;
     };
+    // Up to 16 results: the list lives in registers instead (unsorted; slots >= k hold the largest
+    // value so they never count).  Admitting replaces one entry equal to the current minimum and
+    // takes the minimum again with a compare tree: pure register arithmetic, no chain of
+    // dependent shared-memory round trips.
+    constexpr int KREG = 16;
+    const bool in_regs = k <= KREG;   // warp-uniform
+    uint64_t rl[KREG];
+#pragma unroll
+    for (int i = 0; i < KREG; ++i) rl[i] = (i < k) ? KEY_EMPTY : ~0ull;
+    uint64_t rl_min = KEY_EMPTY;
+    auto admit_regs = [&](uint64_t key) -> uint64_t {
+      bool placed = false;
+#pragma unroll
+      for (int i = 0; i < KREG; ++i) {
+        const bool here = !placed && rl[i] == rl_min;
+        rl[i] = here ? key : rl[i];
+        placed = placed || here;
+      }
+      uint64_t t[KREG];
+#pragma unroll
+      for (int i = 0; i < KREG; ++i) t[i] = rl[i];
+#pragma unroll
+      for (int w2 = KREG / 2; w2 >= 1; w2 /= 2) {
+#pragma unroll
+        for (int i = 0; i < w2; ++i) t[i] = t[i + w2] < t[i] ? t[i + w2] : t[i];
+      }
+      rl_min = t[0];
+      return rl_min;
+    };
     auto drain = [&]() {
       for (int i = 0; i < cnt; ++i) {
         const uint64_t raw = my_queue[i * 32];   // (score bits << 32) | slot
         const uint64_t key = make_key(__uint_as_float((uint32_t)(raw >> 32)), (uint32_t)raw);
         if (key > thr_key) {
-          const uint64_t root = sift_down(key, k);
+          const uint64_t root = in_regs ? admit_regs(key) : sift_down(key, k);
           thr_key = root > thr_floor ? root : thr_floor;
           thr_score = (thr_key == KEY_EMPTY) ? -INFINITY : key_score(thr_key);
         }
@@ -440,13 +469,41 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       }
     }
     if (!ok && lane == 0) report_status(dev_status, DEV_TIMEOUT_MBAR);
-    // sort each private list descending, lanes in parallel: heapsort in place (the smallest
-    // entry goes to the end of the shrinking heap)
-    for (int end = k - 1; end > 0; --end) {
-      const uint64_t smallest = my_list[0];
-      const uint64_t moved = my_list[end * 32];
-      my_list[end * 32] = smallest;
-      sift_down(moved, end);
+    if (in_regs) {
+      // sort the register list descending with a bitonic network (the padding slots >= k hold the
+      // largest value: turn them into the smallest first so that they sort to the end)
+#pragma unroll
+      for (int i = 0; i < KREG; ++i) rl[i] = (i < k) ? rl[i] : KEY_EMPTY;
+#pragma unroll
+      for (int ls = 1; ls <= 4; ++ls) {
+#pragma unroll
+        for (int lj = 3; lj >= 0; --lj) {
+          if (lj < ls) {
+#pragma unroll
+            for (int i = 0; i < KREG; ++i) {
+              const int j = i ^ (1 << lj);
+              if (j > i) {
+                const bool desc = (i & (1 << ls)) == 0;
+                const uint64_t hi = rl[i] > rl[j] ? rl[i] : rl[j], lo = rl[i] > rl[j] ? rl[j] : rl[i];
+                rl[i] = desc ? hi : lo;
+                rl[j] = desc ? lo : hi;
+              }
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < KREG; ++i)
+        if (i < k) my_list[i * 32] = rl[i];
+    } else {
+      // sort each private list descending, lanes in parallel: heapsort in place (the smallest
+      // entry goes to the end of the shrinking heap)
+      for (int end = k - 1; end > 0; --end) {
+        const uint64_t smallest = my_list[0];
+        const uint64_t moved = my_list[end * 32];
+        my_list[end * 32] = smallest;
+        sift_down(moved, end);
+      }
     }
     __syncwarp();
     // transpose out: the partial lists of this warp's queries are contiguous in global memory
