@@ -224,6 +224,10 @@ int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32
     if (out->queue_cap < 1) return fail(IC_ERR_UNSUPPORTED, "tensor-core path: shared memory too small");
     const int fixed = base + QUERY_TILE * out->queue_cap * 8;
     out->n_stages = std::min(8, (smem_optin - fixed) / stage_bytes);
+    if (const char* env = getenv("IC_CACHE_MAX_STAGES")) {   // tuning knob: cap on the ring depth
+      const int cap = atoi(env);
+      if (cap >= 2) out->n_stages = std::min(out->n_stages, cap);
+    }
     if (out->n_stages < 2) return fail(IC_ERR_UNSUPPORTED, "tensor-core path: shared memory too small");
     out->smem_bytes = fixed + out->n_stages * stage_bytes;
     out->n_launches = n_windows * (1 + (out->seed_tiles > 0 ? 1 : 0) + (out->seed0_tiles > 0 ? 1 : 0));

@@ -112,6 +112,8 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int64_t it = 0;
+      int s = 0;          // ring stage and the parity of its current use: plain counters, because a
+      uint32_t ph = 0;    // 64-bit division per K chunk would cost this single thread more than the chunk's MMAs
       bool ok = true;
       // Pacing.  The CTAs (or pairs) that score different query tiles against the same
       // partition read the same row tiles; the tile comes from HBM once only while they stay
@@ -125,8 +127,6 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       for (int64_t tile = tile_begin + part; tile < tile_end && ok; tile += n_part, ++ordinal) {
         if (paced) pace_row[my_unit] = ((unsigned long long)pace_epoch << 32) | ordinal;
         for (int kc = 0; kc < n_kc; ++kc, ++it) {
-          const int s = (int)(it % n_stages);
-          const uint32_t ph = (uint32_t)((it / n_stages) & 1);
           ok = mbar_wait(&tail->empty[s], ph ^ 1u, abort_flag);
           if (!ok) break;
           if (paced && kc == 0) {
@@ -153,13 +153,17 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             tma_load_2d(a_dst, &tmap_q, kc * UM_KC, qt * UM_QT, &tail->full[s]);
             tma_load_2d(a_dst + UM_A_BYTES, &tmap_slab, kc * UM_KC, (int)(tile * UM_RT), &tail->full[s]);
           }
+          if (++s == n_stages) {
+            s = 0;
+            ph ^= 1u;
+          }
         }
       }
       if (!ok) {
         report_status(dev_status, DEV_TIMEOUT_MBAR);
         // loads already issued still write this CTA's shared memory: wait for them (bounded)
         for (int64_t j = (it > n_stages ? it - n_stages : 0); j < it && rank == 0; ++j) {
-          const int s = (int)(j % n_stages);
+          const int s = (int)(j % n_stages);   // (failure path only)
           const long long t0 = clock64();
           while (!mbar_try_wait(&tail->full[s], (uint32_t)((j / n_stages) & 1)) &&
                  clock64() - t0 < WAIT_LIMIT_CYCLES) {
@@ -171,9 +175,11 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0 && rank == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16_f32(UM_QT * CG, UM_RT);
-      int64_t it = 0;
+      int s = 0;          // ring stage and parity as plain counters (see the producer)
+      uint32_t ph = 0;
       int64_t lt = 0;
       bool ok = true;
+      const uint32_t ring_addr = smem_u32(ring);
       for (int64_t tile = tile_begin + part; tile < tile_end && ok; tile += n_part, ++lt) {
         const int buf = (int)(lt & 1);
         const uint32_t bph = (uint32_t)((lt >> 1) & 1);
@@ -181,13 +187,11 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         if (!ok) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * UM_RT);
-        for (int kc = 0; kc < n_kc; ++kc, ++it) {
-          const int s = (int)(it % n_stages);
-          const uint32_t ph = (uint32_t)((it / n_stages) & 1);
+        for (int kc = 0; kc < n_kc; ++kc) {
           ok = mbar_wait(&tail->full[s], ph, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          const uint32_t a_addr = smem_u32(ring + (size_t)s * STAGE_BYTES);
+          const uint32_t a_addr = ring_addr + (uint32_t)(s * STAGE_BYTES);
           const uint64_t da = umma_desc_k_major_sw128(a_addr);
           const uint64_t db = umma_desc_k_major_sw128(a_addr + UM_A_BYTES);
 #pragma unroll
@@ -199,6 +203,10 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           // stage reusable (in both CTAs of a pair) once these MMAs have read it
           if (CG == 2) umma_commit_pair_both(&tail->empty[s]);
           else umma_commit(&tail->empty[s]);
+          if (++s == n_stages) {
+            s = 0;
+            ph ^= 1u;
+          }
         }
         if (ok) {
           if (CG == 2) umma_commit_pair_both(&tail->acc_full[buf]);
