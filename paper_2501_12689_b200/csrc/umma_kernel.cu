@@ -376,19 +376,41 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           thr_score = tau;
         }
       }
+      // Tensor-memory loads take several hundred cycles each while MMAs are running, so the tile
+      // is read 64 columns at a time with two loads in flight, and one vote rejects all 64 columns
+      // in the common case.  Only when some lane has a passing column are the two halves taken
+      // through the admission code below, one after the other.
 #pragma unroll 1
-      for (int cb = 0; cb < UM_RT / 32; ++cb) {
-        uint32_t v[32];
-        tmem_ld_32x32(t_addr + (uint32_t)(cb * 32), v);
+      for (int cp = 0; cp < UM_RT / 64; ++cp) {
+        uint32_t v[32], w[32];
+        tmem_ld_32x32(t_addr + (uint32_t)(cp * 64), v);
+        tmem_ld_32x32(t_addr + (uint32_t)(cp * 64 + 32), w);
         tmem_ld_wait();
-        if (cb == UM_RT / 32 - 1) {
+        if (cp == UM_RT / 64 - 1) {
           // the accumulator has been read completely: hand it back to the MMA issuer
           tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(lead_acc_empty0 + (uint32_t)(buf * 8));
         }
+        if (row0 + cp * 64 + 64 <= n) {   // warp-uniform; a ragged tail goes through the per-half masks
+          float b[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            b[j] = fmaxf(fmaxf(fmaxf(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1])),
+                               fmaxf(__uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]))),
+                         fmaxf(fmaxf(__uint_as_float(w[4 * j]), __uint_as_float(w[4 * j + 1])),
+                               fmaxf(__uint_as_float(w[4 * j + 2]), __uint_as_float(w[4 * j + 3]))));
+          const float best64 = fmaxf(fmaxf(fmaxf(b[0], b[1]), fmaxf(b[2], b[3])), fmaxf(fmaxf(b[4], b[5]), fmaxf(b[6], b[7])));
+          if (!__any_sync(FULL_MASK, best64 >= thr_score)) continue;
+        }
+#pragma unroll 1
+        for (int h = 0; h < 2; ++h) {
+        if (h == 1) {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) v[c] = w[c];
+        }
+        const int cb = cp * 2 + h;
         const int64_t col0 = row0 + cb * 32;
-        const bool last_batch = cb == UM_RT / 32 - 1;
         float g[8];                                   // maxima of the eight groups of four columns
         bool active = col0 < n;                       // warp-uniform
         if (active) {
@@ -469,12 +491,13 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
               need_drain = __any_sync(FULL_MASK, 2 * cnt >= qcap);
             }
           }
-          // fresh thresholds for the next tile
-          if (!active && last_batch) need_drain = need_drain || __any_sync(FULL_MASK, cnt > 0);
           if (need_drain) drain();
           if (!active) break;
         }
+        }   // halves
       }
+      // fresh thresholds for the next tile
+      if (__any_sync(FULL_MASK, cnt > 0)) drain();
     }
     if (!ok && lane == 0) report_status(dev_status, DEV_TIMEOUT_MBAR);
     if (in_regs) {
