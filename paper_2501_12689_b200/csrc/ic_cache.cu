@@ -83,7 +83,7 @@ struct ic_cache {
   bool own_slab = false;
   int64_t* ids = nullptr;
   bool own_ids = false;
-  Buffer q_bf16, q_f32, partials, thr, pace, stage_in, stage_ids, stage_scores, evict;
+  Buffer q_bf16, q_f32, partials, thr, maxima, pace, stage_in, stage_ids, stage_scores, evict;
   unsigned pace_epoch = 0;
   int l2_bytes = 0;
   int* h_status = nullptr;  // pinned, mapped; kernels write a code when a bounded wait expires
@@ -199,22 +199,27 @@ int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32
     const int units = out->n_query_tiles / out->cta_group;                    // CTAs or pairs per partition
     out->n_partitions = std::max(1, std::min((sm_count / out->cta_group) / units, merge_lists_max - 1));
     out->n_ctas = out->n_partitions * out->n_query_tiles;
-    // Threshold seeding: with enough row tiles per CTA, first score 1/16 of them, merge that
-    // sample's lists into its exact top-k and start the main pass from the sample's k-th key.
+    // Threshold seeding, with enough row tiles per CTA.  Level 0 (seed0_tiles): a maxima-only
+    // launch over about one tile per SM gives, per query, the k-th largest of the group maxima,
+    // a floor for its top-k; those tiles are scored again by the next launch.  Level 1
+    // (seed_tiles, large caches only): 1/16 of the tiles are scored with that floor into real
+    // lists, whose merge gives the sample's exact k-th key as the floor of the main pass, which
+    // then skips the sampled tiles.
     const int64_t n_tiles = (n + ROW_TILE - 1) / ROW_TILE;
     const char* seed_env = getenv("IC_CACHE_SEED");   // tuning knob: "0" scores everything in one pass
     const bool seeding = !(seed_env && seed_env[0] == '0' && seed_env[1] == 0);
-    if (seeding && n_tiles >= (int64_t)SEED_MIN_TILES_PER_CTA * out->n_partitions) {
+    const int t0 = (sm_count + out->n_partitions - 1) / out->n_partitions;   // level-0 tiles per partition
+    const int64_t level0 = (int64_t)t0 * out->n_partitions;
+    if (seeding && n_tiles >= (int64_t)SEED_MIN_TILES_PER_CTA * out->n_partitions && n / ROW_TILE >= level0 &&
+        level0 * 4 >= k && level0 * 4 <= 1280) {
+      out->seed0_tiles = (int32_t)level0;
       int seed_fraction = SEED_FRACTION;
       if (const char* fe = getenv("IC_CACHE_SEED_FRACTION")) {   // tuning knob: 1/fraction of the tiles are sampled
         const int f = atoi(fe);
         if (f >= 2) seed_fraction = f;
       }
       const int64_t t = n_tiles / seed_fraction / out->n_partitions * out->n_partitions;
-      out->seed_tiles = (int32_t)std::max<int64_t>(out->n_partitions, t);
-      // with several tiles per CTA in that sample, seed the sample itself from one tile per CTA
-      if (out->seed_tiles >= SEED_TWO_LEVEL_TILES_PER_CTA * out->n_partitions)
-        out->seed0_tiles = std::max(out->n_partitions, out->seed_tiles / 16 / out->n_partitions * out->n_partitions);
+      if (t >= (int64_t)SEED_TWO_LEVEL_TILES_PER_CTA * out->n_partitions && t > level0) out->seed_tiles = (int32_t)t;
     }
     // 1 KiB alignment slack + 256 B of barriers, the per-query lists, then as many candidate
     // queue entries per query (up to 8) as still leave room for two ring stages
@@ -267,15 +272,15 @@ int do_insert(ic_cache* c, const void* emb, const int64_t* ids, int64_t n) {
   return IC_OK;
 }
 
-// Tensor-core scoring of one window: up to two threshold-seeding passes over growing samples of
-// the row tiles, each followed by a merge of its lists (plus the previous sample's merged list)
-// into the sample's exact top-k, then the main pass over the remaining tiles starting from
-// the last sample's k-th key.  Lists are blocks of nq*k keys inside `partials`:
-//   blocks 0 .. P-1      main pass            block P          last merged sample list
-//   blocks P+1 .. 2P     lists of a seeding pass                block 2P+1   first sample's merged list
+// Tensor-core scoring of one window: an optional maxima-only launch over seed0_tiles tiles whose
+// group maxima give a first floor per query (select kernel), an optional launch over the first
+// seed_tiles tiles into real lists whose merge gives the sample's exact k-th key, then the main
+// pass over the tiles not yet in a list.  Lists are blocks of nq*k keys inside `partials`:
+//   blocks 0 .. P-1      main pass            block P          merged sample list
+//   blocks P+1 .. 2P     lists of the sampling launch
 // On return *n_final_lists tells the final merge how many leading blocks to read.
 int run_umma_passes(ic_cache* c, const ic_cache_plan_t& pl, const void* q_bf16, int nq, int nq_pad, int k,
-                    uint64_t* partials, uint64_t* thr, unsigned long long* pace, int* n_final_lists,
+                    uint64_t* partials, uint64_t* thr, float* maxima, unsigned long long* pace, int* n_final_lists,
                     bool profile) {
   if (!c->have_tmap_slab) return fail(IC_ERR_UNSUPPORTED, "tensor-core path unavailable: no tensor map for the slab");
   const int P = pl.n_partitions;
@@ -308,34 +313,46 @@ int run_umma_passes(ic_cache* c, const ic_cache_plan_t& pl, const void* q_bf16, 
     else up.pace_window = w;
   }
   const int64_t n_tiles = (c->size + ROW_TILE - 1) / ROW_TILE;
-  const int64_t bounds[3] = {pl.seed0_tiles, pl.seed_tiles, n_tiles};   // ends of pass 0, pass 1, main
   uint64_t* pass_lists = partials + (size_t)(P + 1) * list_block;
-  uint64_t* first_merged = partials + (size_t)(2 * P + 1) * list_block;
-  uint64_t* last_merged = partials + (size_t)P * list_block;
-  int64_t begin = 0;
+  uint64_t* merged = partials + (size_t)P * list_block;
   bool have_thr = false;
+  int64_t begin = 0;
   *n_final_lists = P;
-  for (int level = 0; level < 2; ++level) {
-    const int64_t end = bounds[level];
-    if (end <= begin) continue;   // this seeding level is not used
-    up.tile_begin = begin;
-    up.tile_end = end;
+  cudaError_t e;
+  if (pl.seed0_tiles > 0 && maxima) {
+    up.tile_begin = 0;
+    up.tile_end = pl.seed0_tiles;
+    up.thr_floor = nullptr;
+    up.partials = nullptr;
+    up.maxima_out = maxima;
+    up.pace_epoch = ++c->pace_epoch;
+    if (profile) profile_mark(c, c->ev_seed, c->n_ev_seed);
+    e = icc::launch_umma(up, c->stream);
+    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core maxima launch failed: %s", cudaGetErrorString(e));
+    c->launches += 1;
+    e = icc::launch_select_floor(maxima, pl.seed0_tiles, nq, k, thr, c->stream);
+    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "floor selection launch failed: %s", cudaGetErrorString(e));
+    c->launches += 1;
+    if (profile) profile_mark(c, c->ev_seed, c->n_ev_seed);
+    have_thr = true;   // the tiles themselves are scored again below
+  }
+  up.maxima_out = nullptr;
+  if (pl.seed_tiles > 0) {
+    up.tile_begin = 0;
+    up.tile_end = pl.seed_tiles;
     up.thr_floor = have_thr ? thr : nullptr;
     up.partials = pass_lists;
     up.pace_epoch = ++c->pace_epoch;
     if (profile) profile_mark(c, c->ev_seed, c->n_ev_seed);
-    cudaError_t e = icc::launch_umma(up, c->stream);
-    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core seeding launch failed: %s", cudaGetErrorString(e));
+    e = icc::launch_umma(up, c->stream);
+    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core sampling launch failed: %s", cudaGetErrorString(e));
     c->launches += 1;
-    const bool last_seed = (end == pl.seed_tiles);
-    // pass lists (P blocks) are followed by the first sample's merged list when there is one
-    e = icc::launch_merge_keys(pass_lists, have_thr ? P + 1 : P, nq, k, last_seed ? last_merged : first_merged, thr,
-                               c->stream);
-    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "seed merge launch failed: %s", cudaGetErrorString(e));
+    e = icc::launch_merge_keys(pass_lists, P, nq, k, merged, thr, c->stream);
+    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "sample merge launch failed: %s", cudaGetErrorString(e));
     c->launches += 1;
     if (profile) profile_mark(c, c->ev_seed, c->n_ev_seed);
     have_thr = true;
-    begin = end;
+    begin = pl.seed_tiles;
     *n_final_lists = P + 1;
   }
   up.tile_begin = begin;
@@ -344,7 +361,7 @@ int run_umma_passes(ic_cache* c, const ic_cache_plan_t& pl, const void* q_bf16, 
   up.partials = partials;
   up.pace_epoch = ++c->pace_epoch;
   if (profile) profile_mark(c, c->ev_score, c->n_ev_score);
-  cudaError_t e = icc::launch_umma(up, c->stream);
+  e = icc::launch_umma(up, c->stream);
   if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core scoring launch failed: %s", cudaGetErrorString(e));
   c->launches += 1;
   if (profile) profile_mark(c, c->ev_score, c->n_ev_score);
@@ -364,6 +381,7 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
   const size_t list_block = (size_t)nq * k;   // keys of one partition
   if ((rc = ensure(c, c->partials, (size_t)(2 * pl.n_partitions + 2) * list_block * 8, "partial top-k lists")) != IC_OK) return rc;
   if ((rc = ensure(c, c->thr, (size_t)nq * 8, "seed thresholds")) != IC_OK) return rc;
+  if ((rc = ensure(c, c->maxima, (size_t)pl.seed0_tiles * nq * 16, "group maxima")) != IC_OK) return rc;
 
   cudaError_t e = icc::launch_convert_rows(q, c->input_dtype == IC_F32, nq, c->dim, c->normalize, c->q_bf16.p,
                                            static_cast<float*>(c->q_f32.p), nq_pad, nullptr, nullptr, c->stream);
@@ -403,7 +421,8 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
     }
   } else {
     rc = run_umma_passes(c, pl, c->q_bf16.p, nq, nq_pad, k, partials, static_cast<uint64_t*>(c->thr.p),
-                         static_cast<unsigned long long*>(c->pace.p), &n_final_lists, true);
+                         static_cast<float*>(c->maxima.p), static_cast<unsigned long long*>(c->pace.p), &n_final_lists,
+                         true);
     if (rc != IC_OK) return rc;
   }
   if (pl.path != IC_PATH_UMMA) profile_mark(c, c->ev_score, c->n_ev_score);
@@ -456,7 +475,8 @@ int do_query_window_static(ic_cache* c, const void* q, int nq, int k, int64_t* o
   const size_t off_qf32 = off_qbf16 + round_up((size_t)nq_pad * c->dim * 2);
   const size_t off_part = off_qf32 + round_up((size_t)nq * c->dim * 4);
   const size_t off_thr = off_part + round_up((size_t)(2 * pl.n_partitions + 2) * list_block * 8);
-  const size_t off_pace = off_thr + round_up((size_t)nq * 8);
+  const size_t off_max = off_thr + round_up((size_t)nq * 8);
+  const size_t off_pace = off_max + round_up((size_t)pl.seed0_tiles * nq * 16);
   const size_t need = off_pace + PACE_BYTES;
   if (need > (size_t)IC_STATIC_SCRATCH_BYTES)
     return fail(IC_ERR_NOMEM, "query needs %zu bytes of scratch but the static scratch holds %u; use ic_cache_query or a smaller nq/k",
@@ -467,6 +487,7 @@ int do_query_window_static(ic_cache* c, const void* q, int nq, int k, int64_t* o
   float* q_f32 = reinterpret_cast<float*>(base + off_qf32);
   uint64_t* partials = reinterpret_cast<uint64_t*>(base + off_part);
   uint64_t* thr = reinterpret_cast<uint64_t*>(base + off_thr);
+  float* maxima = reinterpret_cast<float*>(base + off_max);
   unsigned long long* pace = reinterpret_cast<unsigned long long*>(base + off_pace);
 
   cudaError_t e = icc::launch_convert_rows(q, c->input_dtype == IC_F32, nq, c->dim, c->normalize, q_bf16, q_f32, nq_pad,
@@ -503,7 +524,7 @@ int do_query_window_static(ic_cache* c, const void* q, int nq, int k, int64_t* o
       c->launches += 1;
     }
   } else {
-    rc = run_umma_passes(c, pl, q_bf16, nq, nq_pad, k, partials, thr, pace, &n_final_lists, false);
+    rc = run_umma_passes(c, pl, q_bf16, nq, nq_pad, k, partials, thr, maxima, pace, &n_final_lists, false);
     if (rc != IC_OK) return rc;
   }
   e = icc::launch_merge(partials, n_final_lists, nq, k, c->ids, out_ids, out_scores, min_score, out_counts, c->stream);
@@ -705,6 +726,7 @@ void ic_cache_destroy(ic_cache_t* c) {
   release(c->q_f32);
   release(c->partials);
   release(c->thr);
+  release(c->maxima);
   release(c->pace);
   release(c->stage_in);
   release(c->stage_ids);
@@ -924,6 +946,7 @@ int ic_cache_self_similarity(ic_cache_t* c, int64_t first, int64_t count, int64_
     const size_t list_block = (size_t)nq * k;
     if ((rc = ensure(c, c->partials, (size_t)(2 * pl.n_partitions + 2) * list_block * 8, "partial top-k lists")) != IC_OK) return rc;
     if ((rc = ensure(c, c->thr, (size_t)nq * 8, "seed thresholds")) != IC_OK) return rc;
+    if ((rc = ensure(c, c->maxima, (size_t)pl.seed0_tiles * nq * 16, "group maxima")) != IC_OK) return rc;
     uint64_t* partials = static_cast<uint64_t*>(c->partials.p);
     int n_final_lists = 0;
     // the queries are the stored bf16 rows themselves: the query tensor map points into the slab
@@ -933,7 +956,8 @@ int ic_cache_self_similarity(ic_cache_t* c, int64_t first, int64_t count, int64_
     // lanes beyond nq are not real queries, whatever they read)
     const int q_map_rows = (int)std::min<int64_t>((nq + QUERY_TILE - 1) / QUERY_TILE * QUERY_TILE, c->capacity - (first + w0));
     rc = run_umma_passes(c, pl, q_rows, nq, q_map_rows, k, partials, static_cast<uint64_t*>(c->thr.p),
-                         static_cast<unsigned long long*>(c->pace.p), &n_final_lists, false);
+                         static_cast<float*>(c->maxima.p), static_cast<unsigned long long*>(c->pace.p), &n_final_lists,
+                         false);
     if (rc != IC_OK) return rc;
     cudaError_t e = icc::launch_merge(partials, n_final_lists, nq, k, c->ids, out_ids + w0, out_scores + w0, -INFINITY,
                                       nullptr, c->stream, first + w0);

@@ -96,6 +96,8 @@ struct UmmaParams {
   unsigned long long* pace;   // optional [n_part][units per partition] progress words (L2 pacing hint)
   unsigned pace_epoch;        // distinguishes this launch's progress words from older ones
   int pace_window;            // tiles a CTA may run ahead of its slowest sibling
+  float* maxima_out;          // non-NULL: maxima-only launch over full tiles; receives
+                              // [tile - tile_begin][nq][4] group maxima, partials is not written
   int* dev_status;
 };
 cudaError_t launch_umma(const UmmaParams& p, cudaStream_t st);
@@ -113,6 +115,10 @@ cudaError_t launch_merge(const uint64_t* partials, int n_part, int nq, int k, co
 // and out_thr [nq] = the k-th key (KEY_EMPTY when fewer than k candidates exist).
 cudaError_t launch_merge_keys(const uint64_t* partials, int n_part, int nq, int k, uint64_t* out_keys,
                               uint64_t* out_thr, cudaStream_t st);
+// Threshold from group maxima: maxima [n_tiles][nq][4] holds, per query, the best score of
+// n_tiles * 4 disjoint groups of cache rows; out_thr[q] becomes the key floor that admits every
+// score >= the k-th largest of them (KEY_EMPTY when there are fewer than k groups).
+cudaError_t launch_select_floor(const float* maxima, int n_tiles, int nq, int k, uint64_t* out_thr, cudaStream_t st);
 cudaError_t merge_configure(int smem_optin);
 
 }  // namespace icc

@@ -47,13 +47,15 @@ struct UmmaSmemTail {
   int abort_flag;
 };
 
-template <int CG>
+// MAXIMA = true is the maxima-only variant (no candidate lists): a separate instantiation, so that
+// its code costs the list-keeping variant no registers.
+template <int CG, bool MAXIMA>
 __global__ void __launch_bounds__(UM_THREADS, 1)
 umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_slab,
                        int64_t n, int64_t tile_begin, int64_t tile_end, int dim, int nq, int k, int n_query_tiles,
                        int n_part, int n_stages, int qcap, const uint64_t* __restrict__ thr_floor_in,
                        uint64_t* __restrict__ partials, unsigned long long* pace, unsigned pace_epoch,
-                       int pace_window, int* dev_status) {
+                       int pace_window, float* __restrict__ maxima_out, int* dev_status) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   constexpr int STAGE_BYTES = um_stage_bytes<CG>();
@@ -326,6 +328,32 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       tc_fence_after_sync();
       const uint32_t t_addr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * UM_RT);
       const int64_t row0 = tile * UM_RT;
+      if constexpr (MAXIMA) {
+        // Maxima-only launch (full tiles): no candidate lists, just the best score of each group of
+        // 64 cache rows for every query.  The k-th largest of such maxima over all CTAs is a floor
+        // for the top-k (k different rows score at least that much); the rows are scored again,
+        // with that floor, by the launch that follows.
+        float mx[UM_RT / 64];
+#pragma unroll
+        for (int cp = 0; cp < UM_RT / 64; ++cp) {
+          uint32_t v[32], w[32];
+          tmem_ld_32x32(t_addr + (uint32_t)(cp * 64), v);
+          tmem_ld_32x32(t_addr + (uint32_t)(cp * 64 + 32), w);
+          tmem_ld_wait();
+          float b = -INFINITY;
+#pragma unroll
+          for (int c = 0; c < 32; ++c) b = fmaxf(b, fmaxf(__uint_as_float(v[c]), __uint_as_float(w[c])));
+          mx[cp] = b;
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(lead_acc_empty0 + (uint32_t)(buf * 8));
+        if (real)
+          *reinterpret_cast<float4*>(maxima_out + ((size_t)(tile - tile_begin) * nq + q) * 4) =
+              make_float4(mx[0], mx[1], mx[2], mx[3]);
+        continue;
+      }
+      if constexpr (!MAXIMA) {
       if (lt == 0 && thr_floor_in == nullptr && k <= 16 && row0 + UM_RT <= n) {
         // Cold start (empty lists, no seed threshold): read the tile once just to take the
         // maximum of each group of 8 columns.  The k-th largest of the 32 group maxima is a
@@ -498,9 +526,12 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       }
       // fresh thresholds for the next tile
       if (__any_sync(FULL_MASK, cnt > 0)) drain();
+      }   // !MAXIMA
     }
     if (!ok && lane == 0) report_status(dev_status, DEV_TIMEOUT_MBAR);
-    if (in_regs) {
+    if constexpr (MAXIMA) {
+      // nothing to sort or write: this launch produced maxima only
+    } else if (in_regs) {
       // sort the register list descending with a bitonic network (the padding slots >= k hold the
       // largest value: turn them into the smallest first so that they sort to the end)
 #pragma unroll
@@ -540,7 +571,7 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     // transpose out: the partial lists of this warp's queries are contiguous in global memory
     const int q_first = qt * UM_QT + warp * 32;
     const int q_live = min(32, nq - q_first);
-    if (q_live > 0) {
+    if (q_live > 0 && !MAXIMA) {
       uint64_t* dst = partials + ((size_t)part * nq + q_first) * k;
       for (int i = lane; i < q_live * k; i += 32) {
         const int ql = i / k, e = i - ql * k;
@@ -559,10 +590,23 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 }
 
 cudaError_t umma_configure(int smem_optin) {
-  cudaError_t e = cudaFuncSetAttribute(umma_score_topk_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+  cudaError_t e = cudaFuncSetAttribute(umma_score_topk_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(umma_score_topk_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+    e = cudaFuncSetAttribute(umma_score_topk_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(umma_score_topk_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(umma_score_topk_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
   return e;
+}
+
+template <int CG, bool MAXIMA>
+static cudaError_t launch_umma_variant(const UmmaParams& p, cudaStream_t st) {
+  const dim3 grid((unsigned)(p.n_part * p.n_query_tiles));
+  return launch_overlapped(umma_score_topk_kernel<CG, MAXIMA>, grid, dim3(UM_THREADS), (size_t)p.smem_bytes, st, CG, p.tmap_q,
+                           CG == 2 ? p.tmap_slab_half : p.tmap_slab, p.n, p.tile_begin, p.tile_end, p.dim, p.nq, p.k,
+                           p.n_query_tiles, p.n_part, p.n_stages, p.queue_cap, p.thr_floor, p.partials, p.pace,
+                           p.pace_epoch, p.pace_window, p.maxima_out, p.dev_status);
 }
 
 cudaError_t launch_umma(const UmmaParams& p, cudaStream_t st) {
@@ -572,16 +616,13 @@ cudaError_t launch_umma(const UmmaParams& p, cudaStream_t st) {
   const int stage_bytes = p.cta_group == 2 ? um_stage_bytes<2>() : um_stage_bytes<1>();
   const size_t need = 1024 + (size_t)p.n_stages * stage_bytes + (size_t)UM_QT * (p.k + p.queue_cap) * 8 + sizeof(UmmaSmemTail);
   if (need > (size_t)p.smem_bytes) return cudaErrorInvalidValue;
-  const dim3 grid((unsigned)(p.n_part * p.n_query_tiles));
-  if (p.cta_group == 2)
-    return launch_overlapped(umma_score_topk_kernel<2>, grid, dim3(UM_THREADS), (size_t)p.smem_bytes, st, 2, p.tmap_q,
-                             p.tmap_slab_half, p.n, p.tile_begin, p.tile_end, p.dim, p.nq, p.k, p.n_query_tiles, p.n_part,
-                             p.n_stages, p.queue_cap, p.thr_floor, p.partials, p.pace, p.pace_epoch, p.pace_window,
-                             p.dev_status);
-  return launch_overlapped(umma_score_topk_kernel<1>, grid, dim3(UM_THREADS), (size_t)p.smem_bytes, st, 1, p.tmap_q,
-                           p.tmap_slab, p.n, p.tile_begin, p.tile_end, p.dim, p.nq, p.k, p.n_query_tiles, p.n_part,
-                           p.n_stages, p.queue_cap, p.thr_floor, p.partials, p.pace, p.pace_epoch, p.pace_window,
-                           p.dev_status);
+  if (p.maxima_out != nullptr) {
+    // maxima-only launches cover full tiles only
+    if (p.tile_end * UM_RT > p.n) return cudaErrorInvalidValue;
+    return p.cta_group == 2 ? launch_umma_variant<2, true>(p, st) : launch_umma_variant<1, true>(p, st);
+  }
+  if (p.partials == nullptr) return cudaErrorInvalidValue;
+  return p.cta_group == 2 ? launch_umma_variant<2, false>(p, st) : launch_umma_variant<1, false>(p, st);
 }
 
 }  // namespace icc

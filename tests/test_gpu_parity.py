@@ -93,18 +93,19 @@ def test_threshold_seeding_pass(order, nq, k):
 
 @pytest.mark.parametrize("order", ["random", "best_first", "best_last"])
 def test_two_level_threshold_seeding(order):
-    # enough tiles that the sample is itself seeded from a smaller sample first
+    # enough tiles that a sample of them is scored into lists between the maxima launch and the main pass
     _seeding_case(order, 40, 16, 2_600_011, levels=2)
 
 
 def _seeding_case(order, nq, k, n, levels):
-    # enough row tiles per CTA that the tensor-core path scores a sample first and starts the
-    # main pass from the sample's k-th best; with the best rows all inside (or all outside)
-    # the sample, the final merge must still return the exact top-k
+    # enough row tiles per CTA that the tensor-core path takes a floor from a sample first and
+    # starts the main pass from it; with the best rows all inside (or all outside) the sample,
+    # the final merge must still return the exact top-k
     from paper_2501_12689_b200 import ic_cache_plan
     dim = 64
     plan = ic_cache_plan(dim, n, nq, k, IC_PATH_UMMA)
-    assert plan["seed_tiles"] > 0 and (plan["seed0_tiles"] > 0) == (levels == 2)
+    # level 0: maxima-only launch (its tiles are scored again); level 1: a sample scored into lists
+    assert plan["seed0_tiles"] > 0 and (plan["seed_tiles"] > 0) == (levels == 2)
     x, q = _gauss(n, dim, nq, seed=55)
     if order != "random":
         s0 = (x.float() @ q[0].float())
