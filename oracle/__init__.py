@@ -9,5 +9,9 @@ from .ic_oracle import (  # noqa: F401
     f32_to_bf16_bits,
     search,
     self_similarity,
+    kmeans_assign,
+    kmeans_update,
+    kmeans,
+    search_clustered,
 )
 from .check import accept, AcceptanceError  # noqa: F401

@@ -65,6 +65,20 @@ def _load():
         lib.ic_oracle_self_similarity.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_int64,
                                                   ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, ctypes.c_int,
                                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        lib.ic_oracle_kmeans_assign.restype = ctypes.c_int
+        lib.ic_oracle_kmeans_assign.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_int32,
+                                                ctypes.c_void_p, ctypes.c_int32, ctypes.c_int, ctypes.c_void_p,
+                                                ctypes.c_void_p]
+        lib.ic_oracle_kmeans_update.restype = ctypes.c_int
+        lib.ic_oracle_kmeans_update.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_int32,
+                                                ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                                                ctypes.c_void_p, ctypes.c_void_p]
+        lib.ic_oracle_search_clustered.restype = ctypes.c_int
+        lib.ic_oracle_search_clustered.argtypes = [
+            ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p,
+            ctypes.c_int, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p,
+            ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -174,3 +188,93 @@ def self_similarity(x, first: int = 0, count: int | None = None, ids=None, threa
     if rc != 0:
         raise RuntimeError(f"ic_oracle_self_similarity failed with code {rc}")
     return {"ids": out_ids, "scores": out_scores, "slots": out_slots}
+
+
+def kmeans_assign(x, centroids, threads: int | None = None):
+    """Assignment step of K-Means under the cosine metric: for every row of x the centroid (bf16
+    bits, [K,d] uint16) with the largest fp32 dot product, ties to the lower index.
+    Returns (assign int32 [n], best float32 [n])."""
+    lib = _load()
+    x, xdt = _as_matrix(x, "x")
+    c = np.ascontiguousarray(centroids, dtype=np.uint16)
+    n, d = x.shape
+    assign = np.empty((n,), dtype=np.int32)
+    best = np.empty((n,), dtype=np.float32)
+    rc = lib.ic_oracle_kmeans_assign(x.ctypes.data, xdt, n, d, c.ctypes.data, c.shape[0],
+                                     int(threads or default_threads()), assign.ctypes.data, best.ctypes.data)
+    if rc != 0:
+        raise RuntimeError(f"ic_oracle_kmeans_assign failed with code {rc}")
+    return assign, best
+
+
+def kmeans_update(x, assign, centroids_prev):
+    """Update step: every centroid becomes the unit-length mean of its rows (fp64 sums in slot order),
+    rounded to bf16; a centroid without rows keeps its previous value.
+    Returns (centroids uint16 [K,d], exact float64 [K,d], counts int64 [K])."""
+    lib = _load()
+    x, xdt = _as_matrix(x, "x")
+    prev = np.ascontiguousarray(centroids_prev, dtype=np.uint16)
+    a = np.ascontiguousarray(assign, dtype=np.int32)
+    n, d = x.shape
+    k_clusters = prev.shape[0]
+    out = np.empty_like(prev)
+    exact = np.empty((k_clusters, d), dtype=np.float64)
+    counts = np.empty((k_clusters,), dtype=np.int64)
+    rc = lib.ic_oracle_kmeans_update(x.ctypes.data, xdt, n, d, a.ctypes.data, k_clusters, prev.ctypes.data,
+                                     out.ctypes.data, exact.ctypes.data, counts.ctypes.data)
+    if rc != 0:
+        raise RuntimeError(f"ic_oracle_kmeans_update failed with code {rc}")
+    return out, exact, counts
+
+
+def kmeans(x_bits, init_slots, n_iters: int, threads: int | None = None):
+    """Lloyd iteration from the rows at init_slots: n_iters times (assign, update), then one last
+    assignment to the final centroids.  x_bits: bf16 bits [n,d] (what the cache stores).
+    Returns dict(centroids uint16 [K,d], assign int32 [n], best float32 [n])."""
+    x_bits = np.ascontiguousarray(x_bits, dtype=np.uint16)
+    cent = x_bits[np.asarray(init_slots, dtype=np.int64)].copy()
+    for _ in range(n_iters):
+        assign, _best = kmeans_assign(x_bits, cent, threads)
+        cent, _exact, _counts = kmeans_update(x_bits, assign, cent)
+    assign, best = kmeans_assign(x_bits, cent, threads)
+    return {"centroids": cent, "assign": assign, "best": best}
+
+
+def search_clustered(x, q, k: int, centroids, assign, nprobe: int, n_indexed: int | None = None, ids=None,
+                     probes=None, threads: int | None = None, want_all_scores: bool = False):
+    """Two-level retrieval: probe the nprobe closest centroids, search their rows and every row
+    past n_indexed exhaustively.  probes: optional int64 [nq,nprobe] centroid indices to use
+    instead of the centroid step.  Returns dict(ids, scores, slots [nq,k], probes [nq,nprobe],
+    centroid_scores [nq,K], all_scores [nq,n] with -inf for rows not searched, or None)."""
+    lib = _load()
+    x, xdt = _as_matrix(x, "x")
+    q, qdt = _as_matrix(q, "q")
+    c = np.ascontiguousarray(centroids, dtype=np.uint16)
+    n, d = x.shape
+    nq = q.shape[0]
+    n_indexed = n if n_indexed is None else int(n_indexed)
+    a = np.ascontiguousarray(assign, dtype=np.int32)
+    if a.shape[0] < n_indexed:
+        raise ValueError("assign must cover the indexed rows")
+    if ids is not None:
+        ids = np.ascontiguousarray(ids, dtype=np.int64)
+    if probes is not None:
+        probes = np.ascontiguousarray(probes, dtype=np.int64)
+        if probes.shape != (nq, nprobe):
+            raise ValueError("probes must have shape [nq, nprobe]")
+    out_ids = np.empty((nq, k), dtype=np.int64)
+    out_scores = np.empty((nq, k), dtype=np.float32)
+    out_slots = np.empty((nq, k), dtype=np.int64)
+    out_probes = np.empty((nq, nprobe), dtype=np.int64)
+    cscores = np.empty((nq, c.shape[0]), dtype=np.float32)
+    all_scores = np.empty((nq, n), dtype=np.float32) if want_all_scores else None
+    rc = lib.ic_oracle_search_clustered(
+        x.ctypes.data, xdt, ids.ctypes.data if ids is not None else None, n, d, q.ctypes.data, qdt, nq, k,
+        c.ctypes.data, c.shape[0], a.ctypes.data, n_indexed, nprobe,
+        probes.ctypes.data if probes is not None else None, int(threads or default_threads()),
+        out_ids.ctypes.data, out_scores.ctypes.data, out_slots.ctypes.data, out_probes.ctypes.data,
+        cscores.ctypes.data, all_scores.ctypes.data if all_scores is not None else None)
+    if rc != 0:
+        raise RuntimeError(f"ic_oracle_search_clustered failed with code {rc}")
+    return {"ids": out_ids, "scores": out_scores, "slots": out_slots, "probes": out_probes,
+            "centroid_scores": cscores, "all_scores": all_scores}
