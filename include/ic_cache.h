@@ -85,10 +85,12 @@ typedef struct ic_cache_plan {
   int32_t smem_bytes;    /* dynamic shared memory of the scoring kernel                    */
   int32_t n_launches;    /* scoring launches needed for the whole batch                    */
   int32_t queue_cap;     /* tensor-core path: candidate queue entries per query (else 0)   */
-  int32_t seed_tiles;    /* tensor-core path: 256-row tiles scored first to seed the
-                            per-query thresholds of the main pass (0 = single pass)        */
-  int32_t seed0_tiles;   /* tensor-core path: tiles of a first, smaller seeding pass that
-                            seeds the seeding pass itself (0 = none)                       */
+  int32_t seed_tiles;    /* tensor-core path: 256-row tiles scored into lists ahead of the
+                            main pass, whose merged k-th key is the main pass's floor; the
+                            main pass skips them (0 = none)                                */
+  int32_t seed0_tiles;   /* tensor-core path: tiles of a maxima-only launch whose k-th
+                            largest group maximum per query is the first floor; these
+                            tiles are scored again afterwards (0 = none)                   */
   int32_t cta_group;     /* tensor-core path: 2 = CTA pairs issue one 256-query MMA and
                             split each row tile between them, 1 = single CTAs (else 0)     */
 } ic_cache_plan_t;
@@ -216,6 +218,52 @@ int ic_cache_self_similarity(ic_cache_t* c, int64_t first, int64_t count, int64_
  */
 int ic_cache_remove(ic_cache_t* c, const int64_t* ids_host, int64_t n, int64_t* n_removed);
 
+/*
+ * Two-level search (paper Sec. 4.1, "Two-Stage Scalable Example Selection": cached examples
+ * are clustered offline into K groups with K-Means, K = sqrt(N) balancing the K centroid
+ * comparisons against the N/K comparisons inside a cluster; a request is matched to centroids
+ * first and searched inside the closest clusters).
+ *
+ * ic_cache_build_index clusters the entries present at the time of the call.  The paper only
+ * names K-Means; here it is Lloyd iteration under the retrieval metric: an entry belongs to
+ * the centroid with the largest score (ties: lower centroid number), a centroid is the mean of
+ * its entries scaled to unit length and stored as bf16.  n_clusters: 0 = round(sqrt(size)),
+ * else 1 .. min(size, IC_MAX_CLUSTERS).  n_iters >= 0 update steps (0 keeps the initial
+ * centroids).  init_slots_host: HOST array of n_clusters distinct slots whose rows are the
+ * initial centroids, or NULL for slots floor(c * size / n_clusters).  Entries are not moved:
+ * slots, ids and the results of ic_cache_query are unaffected.  Not part of the per-request
+ * path (each iteration scores every entry against every centroid and reads the slab once
+ * more); synchronises the stream.  Replaces any earlier index.  ic_cache_remove and
+ * ic_cache_clear drop the index; entries inserted later stay outside it and are searched
+ * exhaustively by every ic_cache_query_clustered until the index is rebuilt.
+ */
+#define IC_MAX_CLUSTERS 16384
+#define IC_MAX_PROBES 64
+int ic_cache_build_index(ic_cache_t* c, int32_t n_clusters, int32_t n_iters, const int64_t* init_slots_host);
+
+/* Number of clusters of the current index (0 = none) and number of entries it covers.  Either
+ * output may be NULL. */
+int ic_cache_index_info(const ic_cache_t* c, int32_t* n_clusters, int64_t* n_indexed);
+
+/* Copy the index to HOST buffers (inspection and tests): centroids_host [n_clusters, dim] bf16
+ * bit patterns, assign_host [n_indexed] int64 cluster of each indexed slot.  Either may be NULL.
+ * Synchronises the stream.  IC_ERR_INVALID without an index. */
+int ic_cache_read_index(ic_cache_t* c, void* centroids_host, int64_t* assign_host);
+
+/*
+ * ic_cache_query restricted to the entries of the nprobe clusters whose centroids score
+ * highest for the query (ties: lower cluster number) plus every entry inserted after the index
+ * was built.  An approximation of ic_cache_query by design: an entry of the true top-k that
+ * sits in a cluster that is not probed is missed; with nprobe = n_clusters the results are
+ * those of ic_cache_query.  Same argument conventions, ordering and padding as
+ * ic_cache_query.  1 <= nprobe <= IC_MAX_PROBES (clamped to n_clusters); out_probes: optional
+ * device array [nq, nprobe] int64 receiving the probed clusters, best first, -1 padded.
+ * IC_ERR_INVALID without an index.  Work per query: n_clusters + the probed clusters' entries
+ * (about nprobe * size / n_clusters) + the entries inserted since, instead of size.
+ */
+int ic_cache_query_clustered(ic_cache_t* c, const void* q, int32_t nq, int32_t k, int32_t nprobe,
+                             int64_t* out_ids, float* out_scores, int64_t* out_probes);
+
 /* Release the handle and everything the library allocated for it.  NULL is a no-op. */
 void ic_cache_destroy(ic_cache_t* c);
 
@@ -253,9 +301,9 @@ int64_t ic_cache_launch_count(const ic_cache_t* c);
 /*
  * Measurement aid.  While enabled, the launches of this handle are bracketed by pairs of CUDA
  * events on the handle's stream, in three groups: "scoring" = the scan launch(es), or the main
- * pass of the tensor-core path (the launch that reads all rows outside the seeding samples);
- * "seed" = each threshold-seeding pass together with the merge of its lists; "merge" = the
- * final merge.  At most 16384 brackets of each group between two reads; later ones go
+ * pass of the tensor-core path (the launch that reads all rows outside the list-level sample);
+ * "seed" = each threshold-seeding launch together with the selection or merge that turns its
+ * output into per-query floors; "merge" = the final merge.  At most 16384 brackets of each group between two reads; later ones go
  * unrecorded.  ic_cache_query_static records nothing.
  */
 int ic_cache_set_profiling(ic_cache_t* c, int32_t enable);

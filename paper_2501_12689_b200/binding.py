@@ -72,6 +72,11 @@ SIGNATURES = {
     "ic_cache_self_similarity": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
                                                 ctypes.c_void_p]),
     "ic_cache_remove": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.POINTER(ctypes.c_int64)]),
+    "ic_cache_build_index": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]),
+    "ic_cache_index_info": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)]),
+    "ic_cache_read_index": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "ic_cache_query_clustered": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
+                                                ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "ic_cache_destroy": (None, [ctypes.c_void_p]),
     "ic_cache_set_stream": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
     "ic_cache_set_path": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32]),
@@ -294,6 +299,42 @@ class ICCache:
         out_scores = torch.empty(count, dtype=torch.float32, device=self.device)
         _check(load_library().ic_cache_self_similarity(self._h, first, count, _ptr(out_ids), _ptr(out_scores)))
         return out_ids, out_scores
+
+    def build_index(self, n_clusters: int = 0, n_iters: int = 10, init_slots: Optional[torch.Tensor] = None) -> None:
+        """Cluster the current entries (ic_cache_build_index).  init_slots: optional host int64
+        tensor of n_clusters distinct slots whose rows are the initial centroids."""
+        ptr = None
+        if init_slots is not None:
+            if init_slots.dtype != torch.int64 or init_slots.is_cuda or not init_slots.is_contiguous() \
+                    or init_slots.numel() != n_clusters:
+                raise ValueError("init_slots must be a contiguous int64 host tensor with n_clusters entries")
+            ptr = _ptr(init_slots)
+        _check(load_library().ic_cache_build_index(self._h, int(n_clusters), int(n_iters), ptr))
+
+    def index_info(self) -> Tuple[int, int]:
+        """(number of clusters, number of entries the index covers); (0, 0) without an index."""
+        k, n = ctypes.c_int32(0), ctypes.c_int64(0)
+        _check(load_library().ic_cache_index_info(self._h, ctypes.byref(k), ctypes.byref(n)))
+        return int(k.value), int(n.value)
+
+    def read_index(self) -> Tuple[torch.Tensor, torch.Tensor]:
+        """Host copies of the index: (centroids [K, dim] bfloat16, assign [n_indexed] int64)."""
+        k, n = self.index_info()
+        cent = torch.empty(k, self.dim, dtype=torch.bfloat16)
+        assign = torch.empty(n, dtype=torch.int64)
+        _check(load_library().ic_cache_read_index(self._h, _ptr(cent), _ptr(assign)))
+        return cent, assign
+
+    def query_clustered(self, q: torch.Tensor, k: int, nprobe: int, return_probes: bool = False):
+        """Two-level search (ic_cache_query_clustered): (ids, scores) or (ids, scores, probes)."""
+        self._check_rows(q, True, "q")
+        nq = q.shape[0]
+        out_ids = torch.empty(nq, k, dtype=torch.int64, device=self.device)
+        out_scores = torch.empty(nq, k, dtype=torch.float32, device=self.device)
+        probes = torch.empty(nq, nprobe, dtype=torch.int64, device=self.device) if return_probes else None
+        _check(load_library().ic_cache_query_clustered(self._h, _ptr(q), nq, int(k), int(nprobe), _ptr(out_ids),
+                                                       _ptr(out_scores), _ptr(probes) if return_probes else None))
+        return (out_ids, out_scores, probes) if return_probes else (out_ids, out_scores)
 
     def remove(self, ids: torch.Tensor) -> int:
         """Remove every entry whose id is in `ids` (a host int64 tensor); returns how many went."""

@@ -89,6 +89,12 @@ struct ic_cache {
   int* h_status = nullptr;  // pinned, mapped; kernels write a code when a bounded wait expires
   int* d_status = nullptr;
   int64_t launches = 0;
+  // two-level search: the centroids live in a child cache (labels 0 .. n_clusters-1) so that the
+  // ordinary scoring kernels serve both the assignment step and a query's centroid step
+  ic_cache* centroids = nullptr;
+  int32_t n_clusters = 0;
+  int64_t n_indexed = 0;
+  Buffer idx_assign, idx_best, idx_order, idx_offsets, idx_sort, idx_init, idx_probes, idx_probe_scores;
   EncodeTiledFn encode = nullptr;
   CUtensorMap tmap_slab;       // box of 256 rows
   CUtensorMap tmap_slab_half;  // box of 128 rows, for CTA pairs
@@ -533,6 +539,50 @@ int do_query_window_static(ic_cache* c, const void* q, int nq, int k, int64_t* o
   return IC_OK;
 }
 
+// Top-k of `count` stored bf16 rows (q_rows: device, [count, dim]; `readable` rows from q_rows on
+// may be read) against the entries of cache c on the tensor-core path, in windows of 1024 rows.
+// The query tensor map points straight at the rows: no conversion pass.  self_first < 0:
+// out_ids/out_scores are [count, k].  self_first >= 0: the rows are c's own entries from slot
+// self_first on and one result per row is written, its best entry other than itself.
+int query_bf16_rows(ic_cache* c, const char* q_rows, int64_t count, int64_t readable, int k, int64_t* out_ids,
+                    float* out_scores, int64_t self_first) {
+  int rc;
+  for (int64_t w0 = 0; w0 < count; w0 += WINDOW_MAX_NQ) {
+    const int nq = (int)std::min<int64_t>(WINDOW_MAX_NQ, count - w0);
+    ic_cache_plan_t pl;
+    if ((rc = plan_impl(c->dim, c->size, nq, k, IC_PATH_UMMA, c->sm_count, c->smem_optin, &pl)) != IC_OK) return rc;
+    const size_t list_block = (size_t)nq * k;
+    if ((rc = ensure(c, c->partials, (size_t)(2 * pl.n_partitions + 2) * list_block * 8, "partial top-k lists")) != IC_OK) return rc;
+    if ((rc = ensure(c, c->thr, (size_t)nq * 8, "seed thresholds")) != IC_OK) return rc;
+    if ((rc = ensure(c, c->maxima, (size_t)pl.seed0_tiles * nq * 16, "group maxima")) != IC_OK) return rc;
+    uint64_t* partials = static_cast<uint64_t*>(c->partials.p);
+    int n_final_lists = 0;
+    // the map may cover following rows up to a full 128-row tile, never past `readable`; lanes
+    // beyond nq are not real queries, whatever they read
+    const int q_map_rows = (int)std::min<int64_t>((nq + QUERY_TILE - 1) / QUERY_TILE * QUERY_TILE, readable - w0);
+    rc = run_umma_passes(c, pl, q_rows + (size_t)w0 * c->dim * 2, nq, q_map_rows, k, partials,
+                         static_cast<uint64_t*>(c->thr.p), static_cast<float*>(c->maxima.p),
+                         static_cast<unsigned long long*>(c->pace.p), &n_final_lists, false);
+    if (rc != IC_OK) return rc;
+    const size_t out_stride = self_first >= 0 ? 1 : (size_t)k;
+    cudaError_t e = icc::launch_merge(partials, n_final_lists, nq, k, c->ids, out_ids + (size_t)w0 * out_stride,
+                                      out_scores + (size_t)w0 * out_stride, -INFINITY, nullptr, c->stream,
+                                      self_first >= 0 ? self_first + w0 : -1);
+    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "merge launch failed: %s", cudaGetErrorString(e));
+    c->launches += 1;
+  }
+  return IC_OK;
+}
+
+void drop_index(ic_cache* c) {
+  if (c->centroids) {
+    ic_cache_destroy(c->centroids);
+    c->centroids = nullptr;
+  }
+  c->n_clusters = 0;
+  c->n_indexed = 0;
+}
+
 int check_query_args(ic_cache* c, const void* q, int32_t nq, int32_t k, const void* out_ids, const void* out_scores) {
   if (!c) return fail(IC_ERR_INVALID, "NULL handle");
   if (nq < 0) return fail(IC_ERR_INVALID, "nq %d < 0", nq);
@@ -700,6 +750,7 @@ ic_cache_t* ic_cache_create_ex(int32_t dim, int64_t capacity, const ic_cache_opt
     cudaError_t e1 = icc::merge_configure(c->smem_optin);
     cudaError_t e2 = icc::scan_configure(c->smem_optin);
     cudaError_t e3 = icc::umma_configure(c->smem_optin);
+    if (e3 == cudaSuccess) e3 = icc::index_configure(c->smem_optin);
     if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess) {
       cudaGetLastError();
       fail(IC_ERR_CUDA, "kernel attribute set-up failed (merge %d, scan %d, tensor-core %d)", (int)e1, (int)e2, (int)e3);
@@ -720,6 +771,15 @@ void ic_cache_destroy(ic_cache_t* c) {
   if (!c) return;
   DeviceGuard guard(c->device);
   cudaStreamSynchronize(c->stream);
+  drop_index(c);
+  release(c->idx_assign);
+  release(c->idx_best);
+  release(c->idx_order);
+  release(c->idx_offsets);
+  release(c->idx_sort);
+  release(c->idx_init);
+  release(c->idx_probes);
+  release(c->idx_probe_scores);
   if (c->own_slab && c->slab) cudaFree(c->slab);
   if (c->own_ids && c->ids) cudaFree(c->ids);
   release(c->q_bf16);
@@ -924,6 +984,7 @@ int ic_cache_remove(ic_cache_t* c, const int64_t* ids_host, int64_t n, int64_t* 
   }
   c->size = new_size;
   if (n_removed) *n_removed = (int64_t)m;
+  drop_index(c);   // rows moved: member lists and assignments no longer name the right slots
   return IC_OK;
 }
 
@@ -939,30 +1000,166 @@ int ic_cache_self_similarity(ic_cache_t* c, int64_t first, int64_t count, int64_
   int rc = check_timeout(c);
   if (rc != IC_OK) return rc;
   const int k = 2;   // a row's best match is itself or an exact copy; the next one is the answer
-  for (int64_t w0 = 0; w0 < count; w0 += WINDOW_MAX_NQ) {
-    const int nq = (int)std::min<int64_t>(WINDOW_MAX_NQ, count - w0);
-    ic_cache_plan_t pl;
-    if ((rc = plan_impl(c->dim, c->size, nq, k, IC_PATH_UMMA, c->sm_count, c->smem_optin, &pl)) != IC_OK) return rc;
-    const size_t list_block = (size_t)nq * k;
-    if ((rc = ensure(c, c->partials, (size_t)(2 * pl.n_partitions + 2) * list_block * 8, "partial top-k lists")) != IC_OK) return rc;
-    if ((rc = ensure(c, c->thr, (size_t)nq * 8, "seed thresholds")) != IC_OK) return rc;
-    if ((rc = ensure(c, c->maxima, (size_t)pl.seed0_tiles * nq * 16, "group maxima")) != IC_OK) return rc;
-    uint64_t* partials = static_cast<uint64_t*>(c->partials.p);
-    int n_final_lists = 0;
-    // the queries are the stored bf16 rows themselves: the query tensor map points into the slab
-    // (rows past nq read as zero), no conversion pass is needed
-    const char* q_rows = static_cast<const char*>(c->slab) + (size_t)(first + w0) * c->dim * 2;
-    // (the map may cover following slab rows up to a full 128-row tile, never past the slab;
-    // lanes beyond nq are not real queries, whatever they read)
-    const int q_map_rows = (int)std::min<int64_t>((nq + QUERY_TILE - 1) / QUERY_TILE * QUERY_TILE, c->capacity - (first + w0));
-    rc = run_umma_passes(c, pl, q_rows, nq, q_map_rows, k, partials, static_cast<uint64_t*>(c->thr.p),
-                         static_cast<float*>(c->maxima.p), static_cast<unsigned long long*>(c->pace.p), &n_final_lists,
-                         false);
+  const char* q_rows = static_cast<const char*>(c->slab) + (size_t)first * c->dim * 2;
+  return query_bf16_rows(c, q_rows, count, c->capacity - first, k, out_ids, out_scores, first);
+}
+
+int ic_cache_build_index(ic_cache_t* c, int32_t n_clusters, int32_t n_iters, const int64_t* init_slots_host) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  if (c->size < 1) return fail(IC_ERR_INVALID, "cannot cluster an empty cache");
+  if (n_iters < 0) return fail(IC_ERR_INVALID, "n_iters %d < 0", n_iters);
+  const int64_t k_max = std::min<int64_t>(c->size, IC_MAX_CLUSTERS);
+  int64_t K = n_clusters;
+  if (n_clusters == 0) K = std::max<int64_t>(1, std::min<int64_t>(k_max, llround(sqrt((double)c->size))));
+  if (K < 1 || K > k_max) return fail(IC_ERR_INVALID, "n_clusters %d outside [1, %lld]", n_clusters, (long long)k_max);
+  std::vector<int64_t> init((size_t)K);
+  if (init_slots_host) {
+    std::vector<int64_t> sorted(init_slots_host, init_slots_host + K);
+    std::sort(sorted.begin(), sorted.end());
+    for (int64_t i = 0; i < K; ++i) {
+      if (sorted[i] < 0 || sorted[i] >= c->size || (i > 0 && sorted[i] == sorted[i - 1]))
+        return fail(IC_ERR_INVALID, "init_slots must be %lld distinct slots in [0, %lld)", (long long)K, (long long)c->size);
+      init[i] = init_slots_host[i];
+    }
+  } else {
+    for (int64_t i = 0; i < K; ++i) init[i] = i * c->size / K;
+  }
+  DeviceGuard guard(c->device);
+  int rc = check_timeout(c);
+  if (rc != IC_OK) return rc;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(IC_ERR_CUDA, "stream sync failed");
+  drop_index(c);
+  const int64_t n = c->size;
+  if ((rc = ensure(c, c->idx_init, (size_t)K * 8, "initial centroid slots")) != IC_OK) return rc;
+  if ((rc = ensure(c, c->idx_assign, (size_t)n * 8, "cluster assignments")) != IC_OK) return rc;
+  if ((rc = ensure(c, c->idx_best, (size_t)n * 4, "assignment scores")) != IC_OK) return rc;
+  if ((rc = ensure(c, c->idx_order, (size_t)n * 4, "cluster member lists")) != IC_OK) return rc;
+  if ((rc = ensure(c, c->idx_offsets, (size_t)(K + 1) * 4, "cluster offsets")) != IC_OK) return rc;
+  if ((rc = ensure(c, c->idx_sort, icc::sort_scratch_ints(n, (int)K) * 4, "sort scratch")) != IC_OK) return rc;
+  // the child shares device, stream and input conventions, so a query's centroid step sees the
+  // same bf16-rounded query as the scan of the clusters
+  ic_cache_opts_t o;
+  memset(&o, 0, sizeof o);
+  o.struct_size = sizeof o;
+  o.device = c->device;
+  o.input_dtype = c->input_dtype;
+  o.normalize = c->normalize;
+  o.stream = c->stream;
+  ic_cache* child = ic_cache_create_ex(c->dim, K, &o);
+  if (!child) return IC_ERR_NOMEM;   // message already set
+  cudaError_t e = cudaMemcpyAsync(c->idx_init.p, init.data(), (size_t)K * 8, cudaMemcpyHostToDevice, c->stream);
+  if (e == cudaSuccess)
+    e = icc::launch_gather_rows(c->slab, static_cast<const int64_t*>(c->idx_init.p), (int)K, c->dim, child->slab,
+                                child->ids, c->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);   // `init` is a host vector about to go away
+  if (e != cudaSuccess) {
+    ic_cache_destroy(child);
+    return fail(IC_ERR_CUDA, "centroid seeding failed: %s", cudaGetErrorString(e));
+  }
+  child->size = K;
+  child->launches += 1;
+  int64_t* assign = static_cast<int64_t*>(c->idx_assign.p);
+  for (int it = 0; it <= n_iters && rc == IC_OK; ++it) {
+    // assignment: every cached row is a query against the centroids, best centroid per row
+    rc = query_bf16_rows(child, static_cast<const char*>(c->slab), n, c->capacity, 1, assign,
+                         static_cast<float*>(c->idx_best.p), -1);
+    if (rc != IC_OK) break;
+    e = icc::launch_sort_by_cluster(assign, n, (int)K, static_cast<int*>(c->idx_sort.p),
+                                    static_cast<int*>(c->idx_offsets.p), static_cast<int*>(c->idx_order.p), c->stream);
+    if (e == cudaSuccess && it < n_iters)
+      e = icc::launch_centroid_update(c->slab, c->dim, static_cast<const int*>(c->idx_offsets.p),
+                                      static_cast<const int*>(c->idx_order.p), (int)K, child->slab, c->stream);
+    if (e != cudaSuccess) rc = fail(IC_ERR_CUDA, "clustering launch failed: %s", cudaGetErrorString(e));
+    child->launches += it < n_iters ? 5 : 4;
+  }
+  if (rc == IC_OK && cudaStreamSynchronize(c->stream) != cudaSuccess) rc = fail(IC_ERR_CUDA, "clustering failed on the device");
+  if (rc == IC_OK) rc = check_timeout(c);
+  if (rc != IC_OK) {
+    char keep[sizeof g_err];
+    memcpy(keep, g_err, sizeof keep);
+    ic_cache_destroy(child);
+    memcpy(g_err, keep, sizeof keep);
+    return rc;
+  }
+  c->centroids = child;
+  c->n_clusters = (int32_t)K;
+  c->n_indexed = n;
+  return IC_OK;
+}
+
+int ic_cache_index_info(const ic_cache_t* c, int32_t* n_clusters, int64_t* n_indexed) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  if (n_clusters) *n_clusters = c->n_clusters;
+  if (n_indexed) *n_indexed = c->n_indexed;
+  return IC_OK;
+}
+
+int ic_cache_read_index(ic_cache_t* c, void* centroids_host, int64_t* assign_host) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  if (!c->centroids) return fail(IC_ERR_INVALID, "no index: call ic_cache_build_index first");
+  DeviceGuard guard(c->device);
+  cudaError_t e = cudaStreamSynchronize(c->stream);
+  if (e == cudaSuccess && centroids_host)
+    e = cudaMemcpy(centroids_host, c->centroids->slab, (size_t)c->n_clusters * c->dim * 2, cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess && assign_host)
+    e = cudaMemcpy(assign_host, c->idx_assign.p, (size_t)c->n_indexed * 8, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "index copy failed: %s", cudaGetErrorString(e));
+  return IC_OK;
+}
+
+int ic_cache_query_clustered(ic_cache_t* c, const void* q, int32_t nq, int32_t k, int32_t nprobe, int64_t* out_ids,
+                             float* out_scores, int64_t* out_probes) {
+  int rc = check_query_args(c, q, nq, k, out_ids, out_scores);
+  if (rc != IC_OK || nq == 0) return rc;
+  if (!c->centroids) return fail(IC_ERR_INVALID, "no index: call ic_cache_build_index first");
+  if (nprobe < 1 || nprobe > IC_MAX_PROBES) return fail(IC_ERR_INVALID, "nprobe %d outside [1, %d]", nprobe, IC_MAX_PROBES);
+  DeviceGuard guard(c->device);
+  if (!is_device_ptr(q, c->device) || !is_device_ptr(out_ids, c->device) || !is_device_ptr(out_scores, c->device) ||
+      (out_probes && !is_device_ptr(out_probes, c->device)))
+    return fail(IC_ERR_INVALID, "q, out_ids, out_scores and out_probes must be device pointers on device %d", c->device);
+  if ((rc = check_timeout(c)) != IC_OK) return rc;
+  const int np = nprobe;   // probes past the number of clusters come back as -1 and give empty lists
+  const int64_t tail = c->size - c->n_indexed;
+  const size_t q_row = (size_t)c->dim * in_elem_bytes(c);
+  const int merge_lists_max = (c->smem_optin - 4096) / (k * 8 + 4);
+  for (int q0 = 0; q0 < nq; q0 += WINDOW_MAX_NQ) {
+    const int w = std::min(WINDOW_MAX_NQ, nq - q0);
+    const char* qw = static_cast<const char*>(q) + (size_t)q0 * q_row;
+    // pieces per probed cluster: enough CTAs to fill the GPU at small batches, pieces of at least
+    // ~64 rows; the rows inserted since the build are cut into pieces of ~2048
+    const int64_t avg_cluster = std::max<int64_t>(1, c->n_indexed / c->n_clusters);
+    int n_split = (int)std::max<int64_t>(1, std::min<int64_t>({8, (2 * c->sm_count + (int64_t)w * np - 1) / ((int64_t)w * np),
+                                                                avg_cluster / 64}));
+    int n_tail = tail > 0 ? (int)std::max<int64_t>(1, std::min<int64_t>(32, (tail + 2047) / 2048)) : 0;
+    while (np * n_split + n_tail > merge_lists_max && n_split > 1) --n_split;
+    if (np * n_split + n_tail > merge_lists_max) n_tail = std::min(n_tail, std::max(tail > 0 ? 1 : 0, merge_lists_max - np * n_split));
+    if (np * n_split + n_tail > merge_lists_max)
+      return fail(IC_ERR_UNSUPPORTED, "nprobe %d with k %d needs more partial lists than the merge kernel holds", nprobe, k);
+    const int n_lists = np * n_split + n_tail;
+    if ((rc = ensure(c, c->idx_probes, (size_t)w * nprobe * 8, "probed clusters")) != IC_OK) return rc;
+    if ((rc = ensure(c, c->idx_probe_scores, (size_t)w * nprobe * 4, "centroid scores")) != IC_OK) return rc;
+    const int nq_pad = (w + QUERY_TILE - 1) / QUERY_TILE * QUERY_TILE;
+    if ((rc = ensure(c, c->q_bf16, (size_t)nq_pad * c->dim * 2, "query staging (bf16)")) != IC_OK) return rc;
+    if ((rc = ensure(c, c->q_f32, (size_t)w * c->dim * 4, "query staging (fp32)")) != IC_OK) return rc;
+    if ((rc = ensure(c, c->partials, (size_t)n_lists * w * k * 8, "partial top-k lists")) != IC_OK) return rc;
+    // centroid step: the nprobe best centroids of every query (labels = cluster numbers); past
+    // the number of clusters the rows are padded with -1
+    int64_t* probes = out_probes ? out_probes + (size_t)q0 * nprobe : static_cast<int64_t*>(c->idx_probes.p);
+    rc = do_query_window(c->centroids, qw, w, nprobe, probes, static_cast<float*>(c->idx_probe_scores.p), -INFINITY, nullptr);
     if (rc != IC_OK) return rc;
-    cudaError_t e = icc::launch_merge(partials, n_final_lists, nq, k, c->ids, out_ids + w0, out_scores + w0, -INFINITY,
-                                      nullptr, c->stream, first + w0);
-    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "merge launch failed: %s", cudaGetErrorString(e));
-    c->launches += 1;
+    // the same bf16-rounded queries, widened to fp32, for the scan of the clusters
+    cudaError_t e = icc::launch_convert_rows(qw, c->input_dtype == IC_F32, w, c->dim, c->normalize, c->q_bf16.p,
+                                             static_cast<float*>(c->q_f32.p), nq_pad, nullptr, nullptr, c->stream);
+    if (e == cudaSuccess)
+      e = icc::launch_cluster_scan(c->slab, c->size, c->dim, static_cast<const float*>(c->q_f32.p), w, k, probes, nprobe,
+                                   n_split, n_tail, static_cast<const int*>(c->idx_offsets.p),
+                                   static_cast<const int*>(c->idx_order.p), c->n_indexed,
+                                   static_cast<uint64_t*>(c->partials.p), c->stream);
+    if (e == cudaSuccess)
+      e = icc::launch_merge(static_cast<const uint64_t*>(c->partials.p), nprobe * n_split + n_tail, w, k, c->ids,
+                            out_ids + (size_t)q0 * k, out_scores + (size_t)q0 * k, -INFINITY, nullptr, c->stream);
+    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "two-level search launch failed: %s", cudaGetErrorString(e));
+    c->launches += 3;
   }
   return IC_OK;
 }
@@ -979,6 +1176,7 @@ int ic_cache_probe_wait_limit(ic_cache_t* c) {
 int ic_cache_set_stream(ic_cache_t* c, void* cuda_stream) {
   if (!c) return fail(IC_ERR_INVALID, "NULL handle");
   c->stream = static_cast<cudaStream_t>(cuda_stream);
+  if (c->centroids) c->centroids->stream = c->stream;
   return IC_OK;
 }
 
@@ -997,6 +1195,10 @@ int64_t ic_cache_size(const ic_cache_t* c) {
 int ic_cache_clear(ic_cache_t* c) {
   if (!c) return fail(IC_ERR_INVALID, "NULL handle");
   c->size = 0;
+  if (c->centroids) {
+    DeviceGuard guard(c->device);
+    drop_index(c);   // (synchronises the stream)
+  }
   return IC_OK;
 }
 
@@ -1052,7 +1254,7 @@ int ic_cache_read_profile(ic_cache_t* c, double* scoring_ms, int64_t* scoring_la
 
 int64_t ic_cache_launch_count(const ic_cache_t* c) {
   if (!c) return fail(IC_ERR_INVALID, "NULL handle");
-  return c->launches;
+  return c->launches + (c->centroids ? c->centroids->launches : 0);
 }
 
 }  // extern "C"

@@ -121,4 +121,26 @@ cudaError_t launch_merge_keys(const uint64_t* partials, int n_part, int nq, int 
 cudaError_t launch_select_floor(const float* maxima, int n_tiles, int nq, int k, uint64_t* out_thr, cudaStream_t st);
 cudaError_t merge_configure(int smem_optin);
 
+// ---- two-level search (index_kernels.cu)
+constexpr int IC_INDEX_MAX_CLUSTERS = 16384;   // must equal IC_MAX_CLUSTERS; bounds the sort kernels' shared memory
+cudaError_t index_configure(int smem_optin);
+// Rows slots[c] of the slab become rows c of out_rows, labelled c.
+cudaError_t launch_gather_rows(const void* slab, const int64_t* slots, int n_rows, int dim, void* out_rows,
+                               int64_t* out_ids, cudaStream_t st);
+// Stable counting sort of rows 0 .. n-1 by assign[row] in [0, n_clusters): offsets[n_clusters+1]
+// and order[n] (members of cluster c are order[offsets[c] .. offsets[c+1]), ascending slots).
+// scratch must hold sort_scratch_ints(n, n_clusters) ints.
+size_t sort_scratch_ints(int64_t n, int n_clusters);
+cudaError_t launch_sort_by_cluster(const int64_t* assign, int64_t n, int n_clusters, int* scratch, int* offsets,
+                                   int* order, cudaStream_t st);
+// Centroid c (row c of centroids, bf16) becomes the unit-length mean of its member rows.
+cudaError_t launch_centroid_update(const void* slab, int dim, const int* offsets, const int* order, int n_clusters,
+                                   void* centroids, cudaStream_t st);
+// Scores, per query, the rows of its n_probe probed clusters (probes [nq][n_probe], -1 = none),
+// each cut into n_split pieces, and the rows [n_indexed, n) cut into n_tail pieces; writes one
+// sorted partial list per piece: partials [n_probe*n_split + n_tail][nq][k].
+cudaError_t launch_cluster_scan(const void* slab, int64_t n, int dim, const float* q_f32, int nq, int k,
+                                const int64_t* probes, int n_probe, int n_split, int n_tail, const int* offsets,
+                                const int* order, int64_t n_indexed, uint64_t* partials, cudaStream_t st);
+
 }  // namespace icc
