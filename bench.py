@@ -52,6 +52,9 @@ def parse_args():
     ap.add_argument("--no-sweep", action="store_true", help="skip the secondary batch sizes")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--two-level", type=int, default=0, metavar="NPROBE",
+                    help="also build the K-Means index (K = sqrt(N), 5 iterations) and time the two-level search "
+                         "with this many probed clusters, with its recall against the exhaustive result")
     ap.add_argument("--self-similarity-rows", type=int, default=0,
                     help="also time the all-pairs top-1 self-similarity over this many cached rows")
     return ap.parse_args()
@@ -284,6 +287,34 @@ def run_ours(args):
         self_sim = {"rows": rows, "cache_rows": n_now, "ms": ms, "rows_per_sec": rows / (ms * 1e-3),
                     "tflops": 2.0 * rows * n_now * w.dim / (ms * 1e-3) / 1e12}
 
+    two_level = None
+    if args.two_level > 0:
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        cache.build_index(0, 5)
+        cache.sync()
+        build_s = time.perf_counter() - t0
+        k_clusters, n_indexed = cache.index_info()
+        rows = []
+        for q in sorted(set(w.q_sweep) | {nq}):
+            qb = wl.queries(w, q, dev, round_idx=99)
+            exact_ids, _ = cache.query(qb, w.k)
+            for _ in range(3):
+                cache.query_clustered(qb, w.k, args.two_level)
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            reps = 50
+            ev0.record()
+            for _ in range(reps):
+                got_ids, _ = cache.query_clustered(qb, w.k, args.two_level)
+            ev1.record()
+            torch.cuda.synchronize()
+            ms = ev0.elapsed_time(ev1) / reps
+            e, g = exact_ids.cpu().numpy(), got_ids.cpu().numpy()
+            recall = sum(len(set(e[i]) & set(g[i])) for i in range(q)) / float(q * w.k)
+            rows.append({"nq": q, "ms_per_call": ms, "queries_per_sec": q / (ms * 1e-3), "recall_at_k": recall})
+        two_level = {"n_clusters": k_clusters, "n_indexed": n_indexed, "rows_outside_index": cache.size - n_indexed,
+                     "nprobe": args.two_level, "build_s": build_s, "kmeans_iters": 5, "calls": rows}
+
     clocks = sampler.stop() if sampler else None
 
     ms_all, q_all = aggregate_ranks(dist, main["ms"], float(nq * steps))
@@ -363,6 +394,7 @@ def run_ours(args):
         "profiled_region": {"ms_per_step": prof["ms"] / steps},
         "clocks": clocks,
         "self_similarity": self_sim,
+        "two_level": two_level,
         "sweep": [{"nq": r["nq"], "queries_per_sec": r["nq"] * r["steps"] / (r["ms"] * 1e-3),
                    "ms_per_step": r["ms"] / r["steps"], "roofline": roofline_of(r)} for r in sweep],
     }
