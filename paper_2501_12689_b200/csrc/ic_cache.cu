@@ -1125,10 +1125,10 @@ int ic_cache_query_clustered(ic_cache_t* c, const void* q, int32_t nq, int32_t k
   for (int q0 = 0; q0 < nq; q0 += WINDOW_MAX_NQ) {
     const int w = std::min(WINDOW_MAX_NQ, nq - q0);
     const char* qw = static_cast<const char*>(q) + (size_t)q0 * q_row;
-    // pieces per probed cluster: enough CTAs to fill the GPU at small batches, pieces of at least
-    // ~64 rows; the rows inserted since the build are cut into pieces of ~2048
+    // pieces per probed cluster: about six CTAs per SM (the scan is latency-bound per CTA), pieces
+    // of at least ~64 rows; the rows inserted since the build are cut into pieces of ~2048
     const int64_t avg_cluster = std::max<int64_t>(1, c->n_indexed / c->n_clusters);
-    int n_split = (int)std::max<int64_t>(1, std::min<int64_t>({8, (2 * c->sm_count + (int64_t)w * np - 1) / ((int64_t)w * np),
+    int n_split = (int)std::max<int64_t>(1, std::min<int64_t>({16, (6 * c->sm_count + (int64_t)w * np - 1) / ((int64_t)w * np),
                                                                 avg_cluster / 64}));
     int n_tail = tail > 0 ? (int)std::max<int64_t>(1, std::min<int64_t>(32, (tail + 2047) / 2048)) : 0;
     while (np * n_split + n_tail > merge_lists_max && n_split > 1) --n_split;

@@ -252,11 +252,12 @@ cudaError_t launch_centroid_update(const void* slab, int dim, const int* offsets
 // query's n_probe probed clusters (rows named by the cluster's member list); the remaining
 // n_tail lists are pieces of the rows added after the clustering, [n_indexed, n), which every
 // query searches.  One CTA per item: the query sits in shared memory as fp32, each warp takes
-// every 8th pair of rows (two rows in flight per warp), lanes stride over the rows' 16-byte
+// every 8th group of four rows (four rows in flight per warp), lanes stride over the rows' 16-byte
 // chunks, products are accumulated in fp32 and reduced by shuffles.  Each warp keeps a sorted
 // candidate list of its own; at the end warp 0 merges the eight lists into the item's partial
 // list partials[l][q][k].
 constexpr int CS_WARPS = 8;
+constexpr int CS_ROWS = 4;    // rows in flight per warp
 
 __global__ void __launch_bounds__(CS_WARPS * 32)
 cluster_scan_topk_kernel(const __nv_bfloat16* __restrict__ slab, int64_t n, int dim, const float* __restrict__ q_f32,
@@ -296,40 +297,51 @@ cluster_scan_topk_kernel(const __nv_bfloat16* __restrict__ slab, int64_t n, int 
   uint64_t* my_list = lists + (size_t)warp * k;
   uint64_t thr = KEY_EMPTY;
   const int n_chunks = dim >> 3;
-  for (int64_t m = m0 + 2 * warp; m < m1; m += 2 * CS_WARPS) {
-    const bool two = m + 1 < m1;
-    const int64_t slot_a = members ? members[m] : m;
-    const int64_t slot_b = two ? (members ? members[m + 1] : m + 1) : slot_a;
-    const uint4* ra = reinterpret_cast<const uint4*>(slab + slot_a * dim);
-    const uint4* rb = reinterpret_cast<const uint4*>(slab + slot_b * dim);
-    float acc_a = 0.0f, acc_b = 0.0f;
+  for (int64_t m = m0 + CS_ROWS * warp; m < m1; m += CS_ROWS * CS_WARPS) {
+    // CS_ROWS rows per warp and step: all their loads are issued before the first product
+    int64_t slot[CS_ROWS];
+    const uint4* row[CS_ROWS];
+    float acc[CS_ROWS];
+#pragma unroll
+    for (int r = 0; r < CS_ROWS; ++r) {
+      const int64_t mr = m + r < m1 ? m + r : m;   // a missing row repeats the first one and is dropped below
+      slot[r] = members ? (int64_t)members[mr] : mr;
+      row[r] = reinterpret_cast<const uint4*>(slab + slot[r] * dim);
+      acc[r] = 0.0f;
+    }
     for (int ch = lane; ch < n_chunks; ch += 32) {
-      const uint4 va = ld_stream_16B(ra + ch);
-      const uint4 vb = ld_stream_16B(rb + ch);
-      float xa[8], xb[8];
-      bf16x8_to_f32(va, xa);
-      bf16x8_to_f32(vb, xb);
+      uint4 v[CS_ROWS];
+#pragma unroll
+      for (int r = 0; r < CS_ROWS; ++r) v[r] = ld_stream_16B(row[r] + ch);
       const float4 q0 = *reinterpret_cast<const float4*>(qs + 8 * ch);
       const float4 q1 = *reinterpret_cast<const float4*>(qs + 8 * ch + 4);
-      acc_a = fmaf(xa[0], q0.x, acc_a); acc_b = fmaf(xb[0], q0.x, acc_b);
-      acc_a = fmaf(xa[1], q0.y, acc_a); acc_b = fmaf(xb[1], q0.y, acc_b);
-      acc_a = fmaf(xa[2], q0.z, acc_a); acc_b = fmaf(xb[2], q0.z, acc_b);
-      acc_a = fmaf(xa[3], q0.w, acc_a); acc_b = fmaf(xb[3], q0.w, acc_b);
-      acc_a = fmaf(xa[4], q1.x, acc_a); acc_b = fmaf(xb[4], q1.x, acc_b);
-      acc_a = fmaf(xa[5], q1.y, acc_a); acc_b = fmaf(xb[5], q1.y, acc_b);
-      acc_a = fmaf(xa[6], q1.z, acc_a); acc_b = fmaf(xb[6], q1.z, acc_b);
-      acc_a = fmaf(xa[7], q1.w, acc_a); acc_b = fmaf(xb[7], q1.w, acc_b);
+#pragma unroll
+      for (int r = 0; r < CS_ROWS; ++r) {
+        float x[8];
+        bf16x8_to_f32(v[r], x);
+        float a = acc[r];
+        a = fmaf(x[0], q0.x, a);
+        a = fmaf(x[1], q0.y, a);
+        a = fmaf(x[2], q0.z, a);
+        a = fmaf(x[3], q0.w, a);
+        a = fmaf(x[4], q1.x, a);
+        a = fmaf(x[5], q1.y, a);
+        a = fmaf(x[6], q1.z, a);
+        a = fmaf(x[7], q1.w, a);
+        acc[r] = a;
+      }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-      acc_a += __shfl_xor_sync(FULL_MASK, acc_a, o);
-      acc_b += __shfl_xor_sync(FULL_MASK, acc_b, o);
+#pragma unroll
+      for (int r = 0; r < CS_ROWS; ++r) acc[r] += __shfl_xor_sync(FULL_MASK, acc[r], o);
     }
-    const uint64_t key_a = make_key(acc_a, (uint32_t)slot_a);
-    if (key_a > thr) thr = warp_sorted_insert(my_list, k, key_a, lane);
-    if (two) {
-      const uint64_t key_b = make_key(acc_b, (uint32_t)slot_b);
-      if (key_b > thr) thr = warp_sorted_insert(my_list, k, key_b, lane);
+#pragma unroll
+    for (int r = 0; r < CS_ROWS; ++r) {
+      if (m + r < m1) {   // warp-uniform
+        const uint64_t key = make_key(acc[r], (uint32_t)slot[r]);
+        if (key > thr) thr = warp_sorted_insert(my_list, k, key, lane);
+      }
     }
   }
   __syncthreads();
