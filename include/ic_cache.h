@@ -219,6 +219,26 @@ int ic_cache_self_similarity(ic_cache_t* c, int64_t first, int64_t count, int64_
 int ic_cache_remove(ic_cache_t* c, const int64_t* ids_host, int64_t n, int64_t* n_removed);
 
 /*
+ * Per-entry utility for the cache-management policy (paper Sec. 4.3, "Example Manager": each
+ * example's value is the efficiency gain it enabled, i.e. the number of successful offloadings,
+ * kept as a moving average that is multiplied by 0.9 every hour; a knapsack solver run by the
+ * caller decides what to evict).  The library keeps one fp32 utility per entry, 0 for a new entry;
+ * it moves with the entry when ic_cache_remove closes gaps.  The array (4 bytes per slot of
+ * capacity) is allocated by the first ic_cache_utility_add.
+ *
+ * ic_cache_utility_add: for i in 0..n-1, in order, add gains_host[i] (finite) to the utility of
+ * every entry whose id is ids_host[i] (HOST arrays; ids that match nothing are ignored; one fp32
+ * addition per match).  One pass over the id array; synchronises the stream.
+ * ic_cache_utility_decay: multiply every entry's utility by factor (finite, >= 0; 0.9 per hour in
+ * the paper; the caller owns the clock).  Stream-ordered.
+ * ic_cache_utility_read: copy ids and utilities of slots 0 .. size-1 to HOST arrays (either may
+ * be NULL) for the caller's solver, which then calls ic_cache_remove.  Synchronises the stream.
+ */
+int ic_cache_utility_add(ic_cache_t* c, const int64_t* ids_host, const float* gains_host, int64_t n);
+int ic_cache_utility_decay(ic_cache_t* c, float factor);
+int ic_cache_utility_read(ic_cache_t* c, int64_t* ids_host, float* utility_host);
+
+/*
  * Two-level search (paper Sec. 4.1, "Two-Stage Scalable Example Selection": cached examples
  * are clustered offline into K groups with K-Means, K = sqrt(N) balancing the K centroid
  * comparisons against the N/K comparisons inside a cluster; a request is matched to centroids

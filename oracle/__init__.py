@@ -13,5 +13,7 @@ from .ic_oracle import (  # noqa: F401
     kmeans_update,
     kmeans,
     search_clustered,
+    utility_add,
+    utility_decay,
 )
 from .check import accept, AcceptanceError  # noqa: F401

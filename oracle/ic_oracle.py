@@ -278,3 +278,24 @@ def search_clustered(x, q, k: int, centroids, assign, nprobe: int, n_indexed: in
         raise RuntimeError(f"ic_oracle_search_clustered failed with code {rc}")
     return {"ids": out_ids, "scores": out_scores, "slots": out_slots, "probes": out_probes,
             "centroid_scores": cscores, "all_scores": all_scores}
+
+
+def utility_add(entry_ids, utility, add_ids, gains):
+    """Per-entry utility bookkeeping of the cache manager (paper Sec. 4.3, "Example Manager": an
+    example's value is the efficiency gain it enabled, kept as a moving average).  For every pair
+    (add_ids[i], gains[i]), in order, the gain is added (one fp32 addition) to the utility of every
+    entry carrying that id.  Plain loops; returns a new float32 array."""
+    ids = np.asarray(entry_ids, dtype=np.int64)
+    out = np.array(utility, dtype=np.float32, copy=True)
+    for wanted, gain in zip(np.asarray(add_ids, dtype=np.int64).tolist(), np.asarray(gains, dtype=np.float32)):
+        for slot in range(ids.shape[0]):
+            if ids[slot] == wanted:
+                out[slot] = np.float32(out[slot] + gain)
+    return out
+
+
+def utility_decay(utility, factor):
+    """The moving average's decay step (paper Sec. 4.3: a factor of 0.9 every hour): every utility
+    is multiplied by the factor, one fp32 multiplication each."""
+    f = np.float32(factor)
+    return np.array([np.float32(u * f) for u in np.asarray(utility, dtype=np.float32)], dtype=np.float32)

@@ -72,6 +72,9 @@ SIGNATURES = {
     "ic_cache_self_similarity": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
                                                 ctypes.c_void_p]),
     "ic_cache_remove": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.POINTER(ctypes.c_int64)]),
+    "ic_cache_utility_add": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64]),
+    "ic_cache_utility_decay": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_float]),
+    "ic_cache_utility_read": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "ic_cache_build_index": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]),
     "ic_cache_index_info": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)]),
     "ic_cache_read_index": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
@@ -299,6 +302,24 @@ class ICCache:
         out_scores = torch.empty(count, dtype=torch.float32, device=self.device)
         _check(load_library().ic_cache_self_similarity(self._h, first, count, _ptr(out_ids), _ptr(out_scores)))
         return out_ids, out_scores
+
+    def utility_add(self, ids: torch.Tensor, gains: torch.Tensor) -> None:
+        """Add gains[i] to the utility of every entry whose id is ids[i] (host int64 / float32 tensors)."""
+        if ids.dtype != torch.int64 or ids.is_cuda or not ids.is_contiguous() or gains.dtype != torch.float32 \
+                or gains.is_cuda or not gains.is_contiguous() or gains.numel() != ids.numel():
+            raise ValueError("ids (int64) and gains (float32) must be contiguous host tensors of equal length")
+        _check(load_library().ic_cache_utility_add(self._h, _ptr(ids), _ptr(gains), ids.numel()))
+
+    def utility_decay(self, factor: float) -> None:
+        _check(load_library().ic_cache_utility_decay(self._h, float(factor)))
+
+    def utility_read(self) -> Tuple[torch.Tensor, torch.Tensor]:
+        """Host copies (ids int64 [size], utility float32 [size]) in slot order."""
+        n = self.size
+        ids = torch.empty(n, dtype=torch.int64)
+        util = torch.empty(n, dtype=torch.float32)
+        _check(load_library().ic_cache_utility_read(self._h, _ptr(ids), _ptr(util)))
+        return ids, util
 
     def build_index(self, n_clusters: int = 0, n_iters: int = 10, init_slots: Optional[torch.Tensor] = None) -> None:
         """Cluster the current entries (ic_cache_build_index).  init_slots: optional host int64

@@ -94,6 +94,8 @@ struct ic_cache {
   ic_cache* centroids = nullptr;
   int32_t n_clusters = 0;
   int64_t n_indexed = 0;
+  float* utility = nullptr;   // [capacity] per-entry utility, allocated on first use, zero for new entries
+  Buffer util_ids, util_gains;
   Buffer idx_assign, idx_best, idx_order, idx_offsets, idx_sort, idx_init, idx_probes, idx_probe_scores;
   EncodeTiledFn encode = nullptr;
   CUtensorMap tmap_slab;       // box of 256 rows
@@ -274,7 +276,25 @@ int do_insert(ic_cache* c, const void* emb, const int64_t* ids, int64_t n) {
                                            c->ids + c->size, c->stream);
   if (e != cudaSuccess) return fail(IC_ERR_CUDA, "insert kernel launch failed: %s", cudaGetErrorString(e));
   c->launches += 1;
+  if (c->utility) {   // new entries start without utility
+    if (cudaMemsetAsync(c->utility + c->size, 0, (size_t)n * 4, c->stream) != cudaSuccess)
+      return fail(IC_ERR_CUDA, "clearing the new entries' utility failed");
+  }
   c->size += n;
+  return IC_OK;
+}
+
+// The utility side array exists from the first call that needs it; until then every utility is 0.
+int ensure_utility(ic_cache* c) {
+  if (c->utility) return IC_OK;
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&c->utility), (size_t)c->capacity * 4);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->utility, 0, (size_t)c->capacity * 4, c->stream);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    if (c->utility) cudaFree(c->utility);
+    c->utility = nullptr;
+    return fail(IC_ERR_NOMEM, "allocation of the utility array (%zu bytes) failed: %s", (size_t)c->capacity * 4, cudaGetErrorString(e));
+  }
   return IC_OK;
 }
 
@@ -772,6 +792,9 @@ void ic_cache_destroy(ic_cache_t* c) {
   DeviceGuard guard(c->device);
   cudaStreamSynchronize(c->stream);
   drop_index(c);
+  if (c->utility) cudaFree(c->utility);
+  release(c->util_ids);
+  release(c->util_gains);
   release(c->idx_assign);
   release(c->idx_best);
   release(c->idx_order);
@@ -977,7 +1000,7 @@ int ic_cache_remove(ic_cache_t* c, const int64_t* ids_host, int64_t n, int64_t* 
   if (!src.empty()) {
     e = cudaMemcpyAsync(d_src, src.data(), src.size() * 8, cudaMemcpyHostToDevice, c->stream);
     if (e == cudaSuccess) e = cudaMemcpyAsync(d_dst, dst.data(), dst.size() * 8, cudaMemcpyHostToDevice, c->stream);
-    if (e == cudaSuccess) e = icc::launch_move_rows(c->slab, c->ids, d_src, d_dst, (int64_t)src.size(), c->dim, c->stream);
+    if (e == cudaSuccess) e = icc::launch_move_rows(c->slab, c->ids, c->utility, d_src, d_dst, (int64_t)src.size(), c->dim, c->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);   // src/dst are host vectors about to go away
     if (e != cudaSuccess) return fail(IC_ERR_CUDA, "row move failed: %s", cudaGetErrorString(e));
     c->launches += 1;
@@ -1002,6 +1025,67 @@ int ic_cache_self_similarity(ic_cache_t* c, int64_t first, int64_t count, int64_
   const int k = 2;   // a row's best match is itself or an exact copy; the next one is the answer
   const char* q_rows = static_cast<const char*>(c->slab) + (size_t)first * c->dim * 2;
   return query_bf16_rows(c, q_rows, count, c->capacity - first, k, out_ids, out_scores, first);
+}
+
+int ic_cache_utility_add(ic_cache_t* c, const int64_t* ids_host, const float* gains_host, int64_t n) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  if (n < 0) return fail(IC_ERR_INVALID, "n %lld < 0", (long long)n);
+  if (n == 0) return IC_OK;
+  if (!ids_host || !gains_host) return fail(IC_ERR_INVALID, "NULL pointer with n > 0");
+  for (int64_t i = 0; i < n; ++i)
+    if (!(gains_host[i] == gains_host[i]) || fabsf(gains_host[i]) == INFINITY) return fail(IC_ERR_INVALID, "gain %lld is not finite", (long long)i);
+  DeviceGuard guard(c->device);
+  int rc = check_timeout(c);
+  if (rc != IC_OK) return rc;
+  if ((rc = ensure_utility(c)) != IC_OK) return rc;
+  // sort by id, keeping the caller's order among equal ids
+  std::vector<int64_t> perm((size_t)n);
+  for (int64_t i = 0; i < n; ++i) perm[(size_t)i] = i;
+  std::stable_sort(perm.begin(), perm.end(), [&](int64_t a, int64_t b) { return ids_host[a] < ids_host[b]; });
+  std::vector<int64_t> ids((size_t)n);
+  std::vector<float> gains((size_t)n);
+  for (int64_t i = 0; i < n; ++i) {
+    ids[(size_t)i] = ids_host[perm[(size_t)i]];
+    gains[(size_t)i] = gains_host[perm[(size_t)i]];
+  }
+  if ((rc = ensure(c, c->util_ids, (size_t)n * 8, "utility update ids")) != IC_OK) return rc;
+  if ((rc = ensure(c, c->util_gains, (size_t)n * 4, "utility update gains")) != IC_OK) return rc;
+  cudaError_t e = cudaMemcpyAsync(c->util_ids.p, ids.data(), (size_t)n * 8, cudaMemcpyHostToDevice, c->stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(c->util_gains.p, gains.data(), (size_t)n * 4, cudaMemcpyHostToDevice, c->stream);
+  if (e == cudaSuccess)
+    e = icc::launch_utility_add(c->ids, c->size, static_cast<const int64_t*>(c->util_ids.p),
+                                static_cast<const float*>(c->util_gains.p), n, c->utility, c->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);   // the sorted copies are host vectors about to go away
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "utility update failed: %s", cudaGetErrorString(e));
+  c->launches += 1;
+  return IC_OK;
+}
+
+int ic_cache_utility_decay(ic_cache_t* c, float factor) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  if (!(factor >= 0.0f) || factor == INFINITY) return fail(IC_ERR_INVALID, "decay factor must be finite and >= 0");
+  if (!c->utility || c->size == 0) return IC_OK;   // all utilities are zero
+  DeviceGuard guard(c->device);
+  int rc = check_timeout(c);
+  if (rc != IC_OK) return rc;
+  cudaError_t e = icc::launch_utility_scale(c->utility, c->size, factor, c->stream);
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "utility decay launch failed: %s", cudaGetErrorString(e));
+  c->launches += 1;
+  return IC_OK;
+}
+
+int ic_cache_utility_read(ic_cache_t* c, int64_t* ids_host, float* utility_host) {
+  if (!c) return fail(IC_ERR_INVALID, "NULL handle");
+  if (c->size == 0) return IC_OK;
+  DeviceGuard guard(c->device);
+  cudaError_t e = cudaStreamSynchronize(c->stream);
+  if (e == cudaSuccess && ids_host) e = cudaMemcpy(ids_host, c->ids, (size_t)c->size * 8, cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess && utility_host) {
+    if (c->utility) e = cudaMemcpy(utility_host, c->utility, (size_t)c->size * 4, cudaMemcpyDeviceToHost);
+    else memset(utility_host, 0, (size_t)c->size * 4);
+  }
+  if (e != cudaSuccess) return fail(IC_ERR_CUDA, "utility copy failed: %s", cudaGetErrorString(e));
+  return IC_OK;
 }
 
 int ic_cache_build_index(ic_cache_t* c, int32_t n_clusters, int32_t n_iters, const int64_t* init_slots_host) {

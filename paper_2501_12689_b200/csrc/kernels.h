@@ -46,8 +46,14 @@ cudaError_t launch_convert_rows(const void* in, int in_is_f32, int64_t nrows, in
 cudaError_t launch_find_ids(const int64_t* ids, int64_t n, const int64_t* wanted, int64_t n_wanted, int64_t* match_slots,
                             unsigned long long* match_count, int64_t cap, cudaStream_t st);
 // Move rows (and ids) inside the slab, src[i] -> dst[i]; the two sets must be disjoint.
-cudaError_t launch_move_rows(void* slab, int64_t* ids, const int64_t* src, const int64_t* dst, int64_t nmoves, int dim,
-                             cudaStream_t st);
+// (utility: optional per-row fp32 side array that moves along.)
+cudaError_t launch_move_rows(void* slab, int64_t* ids, float* utility, const int64_t* src, const int64_t* dst,
+                             int64_t nmoves, int dim, cudaStream_t st);
+// utility[row] += gains[j] for every j with wanted[j] == ids[row] (wanted sorted ascending; equal
+// ids are added in their order); utility[row] *= factor for all rows.
+cudaError_t launch_utility_add(const int64_t* ids, int64_t n, const int64_t* wanted, const float* gains, int64_t n_wanted,
+                               float* utility, cudaStream_t st);
+cudaError_t launch_utility_scale(float* utility, int64_t n, float factor, cudaStream_t st);
 
 // Diagnostic: a bounded wait that is made to run out after limit_cycles (nothing completes the
 // barrier); the kernel reports DEV_TIMEOUT_MBAR in the status word and returns.

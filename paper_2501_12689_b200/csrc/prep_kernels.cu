@@ -115,8 +115,8 @@ find_ids_kernel(const int64_t* __restrict__ ids, int64_t n, const int64_t* __res
 // Copy whole rows (and their ids) inside the slab: row src[i] -> row dst[i].  The two sets are
 // disjoint (tail rows move into vacated slots), so rows can move in parallel.
 __global__ void __launch_bounds__(CONV_WARPS * 32)
-move_rows_kernel(__nv_bfloat16* __restrict__ slab, int64_t* __restrict__ ids, const int64_t* __restrict__ src,
-                 const int64_t* __restrict__ dst, int64_t nmoves, int dim) {
+move_rows_kernel(__nv_bfloat16* __restrict__ slab, int64_t* __restrict__ ids, float* __restrict__ utility,
+                 const int64_t* __restrict__ src, const int64_t* __restrict__ dst, int64_t nmoves, int dim) {
   grid_dep_launch_dependents();
   grid_dep_wait();
   const int lane = threadIdx.x & 31;
@@ -126,7 +126,10 @@ move_rows_kernel(__nv_bfloat16* __restrict__ slab, int64_t* __restrict__ ids, co
   const uint4* from = reinterpret_cast<const uint4*>(slab + s * dim);
   uint4* to = reinterpret_cast<uint4*>(slab + d * dim);
   for (int c = lane; c < (dim >> 3); c += 32) to[c] = from[c];
-  if (lane == 0) ids[d] = ids[s];
+  if (lane == 0) {
+    ids[d] = ids[s];
+    if (utility) utility[d] = utility[s];
+  }
 }
 
 cudaError_t launch_find_ids(const int64_t* ids, int64_t n, const int64_t* wanted, int64_t n_wanted, int64_t* match_slots,
@@ -137,12 +140,54 @@ cudaError_t launch_find_ids(const int64_t* ids, int64_t n, const int64_t* wanted
                            match_count, cap);
 }
 
-cudaError_t launch_move_rows(void* slab, int64_t* ids, const int64_t* src, const int64_t* dst, int64_t nmoves, int dim,
-                             cudaStream_t st) {
+cudaError_t launch_move_rows(void* slab, int64_t* ids, float* utility, const int64_t* src, const int64_t* dst,
+                             int64_t nmoves, int dim, cudaStream_t st) {
   if (nmoves == 0) return cudaSuccess;
   const unsigned blocks = (unsigned)((nmoves + CONV_WARPS - 1) / CONV_WARPS);
   return launch_overlapped(move_rows_kernel, dim3(blocks), dim3(CONV_WARPS * 32), 0, st, 1,
-                           static_cast<__nv_bfloat16*>(slab), ids, src, dst, nmoves, dim);
+                           static_cast<__nv_bfloat16*>(slab), ids, utility, src, dst, nmoves, dim);
+}
+
+// Per-entry utility (paper Sec. 4.3, "Example Manager": the efficiency gain of an example, kept as
+// a moving average that is decayed over time).  utility_add_kernel: one thread per cache row looks
+// its id up in `wanted` (sorted ascending, equal ids kept in the caller's order) and adds the gains
+// of all matching entries, one fp32 addition each, in that order.  utility_scale_kernel multiplies
+// every entry's utility by one factor.
+__global__ void __launch_bounds__(256)
+utility_add_kernel(const int64_t* __restrict__ ids, int64_t n, const int64_t* __restrict__ wanted,
+                   const float* __restrict__ gains, int64_t n_wanted, float* __restrict__ utility) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int64_t id = ids[i];
+  int64_t lo = 0, hi = n_wanted;
+  while (lo < hi) {
+    const int64_t mid = (lo + hi) >> 1;
+    if (wanted[mid] < id) lo = mid + 1;
+    else hi = mid;
+  }
+  if (lo < n_wanted && wanted[lo] == id) {
+    float u = utility[i];
+    for (; lo < n_wanted && wanted[lo] == id; ++lo) u += gains[lo];
+    utility[i] = u;
+  }
+}
+
+__global__ void __launch_bounds__(256) utility_scale_kernel(float* __restrict__ utility, int64_t n, float factor) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) utility[i] *= factor;
+}
+
+cudaError_t launch_utility_add(const int64_t* ids, int64_t n, const int64_t* wanted, const float* gains, int64_t n_wanted,
+                               float* utility, cudaStream_t st) {
+  if (n == 0 || n_wanted == 0) return cudaSuccess;
+  utility_add_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(ids, n, wanted, gains, n_wanted, utility);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_utility_scale(float* utility, int64_t n, float factor, cudaStream_t st) {
+  if (n == 0) return cudaSuccess;
+  utility_scale_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(utility, n, factor);
+  return cudaGetLastError();
 }
 
 // Exercise of the bounded-wait path: one thread waits, with a short limit, on an mbarrier that

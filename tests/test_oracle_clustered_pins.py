@@ -189,3 +189,29 @@ def test_well_separated_blobs_are_recovered():
     init = np.array([int(np.flatnonzero(z == b)[0]) for b in range(4)])
     km = oracle.kmeans(xb, init, 3)
     assert np.array_equal(km["assign"], z)           # centroid b starts inside blob b and keeps it
+
+
+# ---------------------------------------------------------------- utility bookkeeping (Sec. 4.3)
+
+def test_utility_hand_computed_sequence():
+    ids = np.array([7, 8, 7, 9], dtype=np.int64)          # id 7 is carried by two entries
+    u = np.zeros(4, dtype=np.float32)
+    u = oracle.utility_add(ids, u, [7, 9, 5], [1.0, 2.0, 4.0])   # id 5 matches nothing
+    assert u.tolist() == [1.0, 0.0, 1.0, 2.0]
+    u = oracle.utility_decay(u, 0.5)
+    assert u.tolist() == [0.5, 0.0, 0.5, 1.0]
+    u = oracle.utility_add(ids, u, [9, 9], [0.25, 0.25])          # the same id twice in one call
+    assert u.tolist() == [0.5, 0.0, 0.5, 1.5]
+    # the paper's decay: 0.9 per hour; after one gain of 1 and two hours 0.81 remains
+    v = oracle.utility_decay(oracle.utility_decay(np.array([1.0], dtype=np.float32), 0.9), 0.9)
+    np.testing.assert_allclose(v, [0.81], rtol=1e-6)
+
+
+def test_utility_moving_average_closed_form():
+    # a gain of g every hour, decayed by 0.9 per hour, is the geometric series g (1 - 0.9^h) / 0.1
+    ids = np.array([1], dtype=np.int64)
+    u = np.zeros(1, dtype=np.float32)
+    for h in range(1, 41):
+        u = oracle.utility_decay(u, 0.9)
+        u = oracle.utility_add(ids, u, [1], [3.0])
+        np.testing.assert_allclose(u[0], 3.0 * (1.0 - 0.9 ** h) / 0.1, rtol=1e-5)
