@@ -99,3 +99,39 @@ def test_full_size_workloads_match_the_oracle_on_sampled_queries(loaded):
             newest = wl.labels(w.insert_rows, "cpu", first_slot=loaded.n - w.insert_rows)
             assert torch.all(sc[:m, 0] > 0.99)
             assert all(int(i) in set(newest.tolist()) for i in ids[:m, 0].cpu())
+
+
+def test_two_level_search_at_full_size(loaded):
+    """The two-level search on the clustered workload at its full size (after the streaming inserts
+    of the test above, so part of the cache lies outside the index once more rows are appended):
+    index build with K = sqrt(N), then sampled queries against the oracle's two-level definition
+    on the library's own centroids, assignment and probes."""
+    w = loaded.w
+    if w.name != "clustered":
+        pytest.skip("two-level search is exercised at full size on the clustered workload")
+    c = loaded.cache
+    c.build_index(0, 3)
+    k_clusters, n_indexed = c.index_info()
+    assert k_clusters == round(n_indexed ** 0.5) and n_indexed == loaded.n
+    nq, nprobe = w.q_sweep[0], 4
+    q = wl.queries(w, nq, DEV, round_idx=7, cache=loaded.x)
+    ids, sc, probes = c.query_clustered(q, w.k, nprobe, return_probes=True)
+    exact_ids, _ = c.query(q, w.k)
+    c.sync()
+    cent, assign = c.read_index()
+    sample = [0, 1, nq // 2, nq - 1]
+    xb = np.concatenate(loaded.host_rows)
+    lab = wl.labels(loaded.n).numpy()
+    ref = oracle.search_clustered(xb, wl.as_bits(q[sample]), w.k, wl.as_bits(cent), assign.numpy().astype(np.int32), nprobe,
+                                  probes=probes[sample].cpu().numpy(), ids=lab, want_all_scores=True)
+    # the probes themselves: each must be within tolerance of the oracle's nprobe best centroids
+    cs = ref["centroid_scores"]
+    for j in range(len(sample)):
+        cut = np.sort(cs[j])[::-1][nprobe - 1]
+        assert np.all(cs[j][probes[sample[j]].cpu().numpy()] >= cut - TOL_STRICT)
+    oracle.accept(ids[sample].cpu().numpy(), sc[sample].cpu().numpy(), ref["all_scores"], w.k, ids=lab, tol=TOL_STRICT,
+                  what="clustered two-level [strict]")
+    # queries sit near cluster centres: a few probes recover the exhaustive result
+    e, g = exact_ids.cpu().numpy(), ids.cpu().numpy()
+    recall = np.mean([len(set(e[i]) & set(g[i])) / w.k for i in range(nq)])
+    assert recall > 0.95, recall
