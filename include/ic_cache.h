@@ -159,7 +159,7 @@ int ic_cache_query_host(ic_cache_t* c, const void* q_host, int32_t nq, int32_t k
  * late cudaMalloc fails), or a latency-critical loop whose rules forbid calls that may
  * synchronise the device, which cudaMalloc and cudaFree do.  ic_cache_query grows the
  * library's scratch buffers on the first call of a larger shape; this variant never does.
- * Its scratch (query staging, partial top-k lists, seed thresholds) is carved out of one
+ * Its scratch (query staging, partial top-k lists, seed thresholds, group maxima) is carved out of one
  * fixed array of IC_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that
  * loads the library holds that much memory until the process exits, whether or not this
  * call is ever used.

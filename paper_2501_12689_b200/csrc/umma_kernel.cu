@@ -13,6 +13,8 @@
 //   warp 5     MMA issuer (one thread) and tensor-memory owner
 // Two 256-column accumulators alternate, so the epilogue of one row tile overlaps the MMAs
 // of the next.  CTA (p, t) scores query tile t against row tiles p, p + P, p + 2P, ...
+// A second instantiation (MAXIMA) shares producer and MMA code but only records, per query and
+// tile, the maxima of four groups of 64 rows: the cheap first step of threshold seeding.
 #include <math.h>
 #include <string.h>
 
@@ -353,7 +355,6 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
               make_float4(mx[0], mx[1], mx[2], mx[3]);
         continue;
       }
-      if constexpr (!MAXIMA) {
       if (lt == 0 && thr_floor_in == nullptr && k <= 16 && row0 + UM_RT <= n) {
         // Cold start (empty lists, no seed threshold): read the tile once just to take the
         // maximum of each group of 8 columns.  The k-th largest of the 32 group maxima is a
@@ -433,100 +434,99 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         }
 #pragma unroll 1
         for (int h = 0; h < 2; ++h) {
-        if (h == 1) {
+          if (h == 1) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) v[c] = w[c];
-        }
-        const int cb = cp * 2 + h;
-        const int64_t col0 = row0 + cb * 32;
-        float g[8];                                   // maxima of the eight groups of four columns
-        bool active = col0 < n;                       // warp-uniform
-        if (active) {
-          if (n - col0 < 32) {                        // ragged last tile: columns past n never admit
-#pragma unroll
-            for (int c = 0; c < 32; ++c)
-              if (col0 + c >= n) v[c] = 0x7fc00000u;
+            for (int c = 0; c < 32; ++c) v[c] = w[c];
           }
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            g[j] = fmaxf(fmaxf(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1])),
-                         fmaxf(__uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
-          const float best = fmaxf(fmaxf(fmaxf(g[0], g[1]), fmaxf(g[2], g[3])), fmaxf(fmaxf(g[4], g[5]), fmaxf(g[6], g[7])));
-          active = __any_sync(FULL_MASK, best >= thr_score);   // common case: nothing passes
-        }
-        // Common slow case: every lane's queue has room for all of its passing columns.  One
-        // vote establishes that, one OR-reduction tells which groups of columns anybody needs,
-        // and the pushes are predicated stores: no per-group votes, no divergent branches.
-        bool drain_after = false;
-        if (active) {
-          uint32_t hm = 0;
-#pragma unroll
-          for (int c = 0; c < 32; ++c) hm |= (__uint_as_float(v[c]) >= thr_score) ? (1u << c) : 0u;
-          if (!__any_sync(FULL_MASK, cnt + __popc(hm) > qcap)) {
-            const uint32_t cols = __reduce_or_sync(FULL_MASK, hm);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              if ((cols >> (4 * j)) & 0xfu) {   // warp-uniform
-#pragma unroll
-                for (int c = 4 * j; c < 4 * j + 4; ++c) {
-                  if ((hm >> c) & 1u) {
-                    my_queue[cnt * 32] = ((uint64_t)v[c] << 32) | (uint32_t)(col0 + c);
-                    ++cnt;
-                  }
-                }
-              }
-            }
-            active = false;
-            drain_after = __any_sync(FULL_MASK, 2 * cnt >= qcap);
-          }
-        }
-        // Otherwise (cold start, very loose thresholds): warp-uniform control flow with the queue
-        // drained at one place only (the code stays small and a drain is always entered by all
-        // 32 lanes, each working through its own queue).  Columns are considered in order;
-        // whenever some lane's queue could not take another group of four (or, for queues
-        // shorter than four, another entry) the pass stops, the queues are drained and the pass
-        // resumes at c_next.
-        int c_next = 0;
-        while (true) {
-          bool need_drain = drain_after;
-          drain_after = false;
+          const int cb = cp * 2 + h;
+          const int64_t col0 = row0 + cb * 32;
+          float g[8];                                   // maxima of the eight groups of four columns
+          bool active = col0 < n;                       // warp-uniform
           if (active) {
+            if (n - col0 < 32) {                        // ragged last tile: columns past n never admit
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              if (!need_drain && 4 * j + 3 >= c_next && __any_sync(FULL_MASK, g[j] >= thr_score)) {
+              for (int c = 0; c < 32; ++c)
+                if (col0 + c >= n) v[c] = 0x7fc00000u;
+            }
 #pragma unroll
-                for (int c = 4 * j; c < 4 * j + 4; ++c) {
-                  if (!need_drain && c >= c_next) {
-                    const float s = __uint_as_float(v[c]);
-                    if (s >= thr_score) {
+            for (int j = 0; j < 8; ++j)
+              g[j] = fmaxf(fmaxf(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1])),
+                           fmaxf(__uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
+            const float best = fmaxf(fmaxf(fmaxf(g[0], g[1]), fmaxf(g[2], g[3])), fmaxf(fmaxf(g[4], g[5]), fmaxf(g[6], g[7])));
+            active = __any_sync(FULL_MASK, best >= thr_score);   // common case: nothing passes
+          }
+          // Common slow case: every lane's queue has room for all of its passing columns.  One
+          // vote establishes that, one OR-reduction tells which groups of columns anybody needs,
+          // and the pushes are predicated stores: no per-group votes, no divergent branches.
+          bool drain_after = false;
+          if (active) {
+            uint32_t hm = 0;
+#pragma unroll
+            for (int c = 0; c < 32; ++c) hm |= (__uint_as_float(v[c]) >= thr_score) ? (1u << c) : 0u;
+            if (!__any_sync(FULL_MASK, cnt + __popc(hm) > qcap)) {
+              const uint32_t cols = __reduce_or_sync(FULL_MASK, hm);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                if ((cols >> (4 * j)) & 0xfu) {   // warp-uniform
+#pragma unroll
+                  for (int c = 4 * j; c < 4 * j + 4; ++c) {
+                    if ((hm >> c) & 1u) {
                       my_queue[cnt * 32] = ((uint64_t)v[c] << 32) | (uint32_t)(col0 + c);
                       ++cnt;
                     }
-                    if (qcap < 4 && __any_sync(FULL_MASK, cnt >= qcap)) {
-                      need_drain = true;
-                      c_next = c + 1;
-                    }
                   }
                 }
-                if (!need_drain && qcap >= 4 && __any_sync(FULL_MASK, cnt + 4 > qcap)) {
-                  need_drain = true;
-                  c_next = 4 * j + 4;
-                }
               }
-            }
-            if (!need_drain) {
               active = false;
-              need_drain = __any_sync(FULL_MASK, 2 * cnt >= qcap);
+              drain_after = __any_sync(FULL_MASK, 2 * cnt >= qcap);
             }
           }
-          if (need_drain) drain();
-          if (!active) break;
-        }
+          // Otherwise (cold start, very loose thresholds): warp-uniform control flow with the queue
+          // drained at one place only (the code stays small and a drain is always entered by all
+          // 32 lanes, each working through its own queue).  Columns are considered in order;
+          // whenever some lane's queue could not take another group of four (or, for queues
+          // shorter than four, another entry) the pass stops, the queues are drained and the pass
+          // resumes at c_next.
+          int c_next = 0;
+          while (true) {
+            bool need_drain = drain_after;
+            drain_after = false;
+            if (active) {
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                if (!need_drain && 4 * j + 3 >= c_next && __any_sync(FULL_MASK, g[j] >= thr_score)) {
+#pragma unroll
+                  for (int c = 4 * j; c < 4 * j + 4; ++c) {
+                    if (!need_drain && c >= c_next) {
+                      const float s = __uint_as_float(v[c]);
+                      if (s >= thr_score) {
+                        my_queue[cnt * 32] = ((uint64_t)v[c] << 32) | (uint32_t)(col0 + c);
+                        ++cnt;
+                      }
+                      if (qcap < 4 && __any_sync(FULL_MASK, cnt >= qcap)) {
+                        need_drain = true;
+                        c_next = c + 1;
+                      }
+                    }
+                  }
+                  if (!need_drain && qcap >= 4 && __any_sync(FULL_MASK, cnt + 4 > qcap)) {
+                    need_drain = true;
+                    c_next = 4 * j + 4;
+                  }
+                }
+              }
+              if (!need_drain) {
+                active = false;
+                need_drain = __any_sync(FULL_MASK, 2 * cnt >= qcap);
+              }
+            }
+            if (need_drain) drain();
+            if (!active) break;
+          }
         }   // halves
       }
       // fresh thresholds for the next tile
       if (__any_sync(FULL_MASK, cnt > 0)) drain();
-      }   // !MAXIMA
     }
     if (!ok && lane == 0) report_status(dev_status, DEV_TIMEOUT_MBAR);
     if constexpr (MAXIMA) {

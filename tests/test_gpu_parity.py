@@ -86,7 +86,7 @@ def test_query_tiling(path, nq, k):
 
 
 @pytest.mark.parametrize("order", ["random", "best_first", "best_last"])
-@pytest.mark.parametrize("nq,k", [(8, 10), (130, 64), (130, 128), (5, 128)])
+@pytest.mark.parametrize("nq,k", [(9, 10), (130, 64), (130, 128), (5, 128)])
 def test_threshold_seeding_pass(order, nq, k):
     _seeding_case(order, nq, k, 400_003, levels=1)
 
