@@ -315,6 +315,25 @@ def run_ours(args):
         two_level = {"n_clusters": k_clusters, "n_indexed": n_indexed, "rows_outside_index": cache.size - n_indexed,
                      "nprobe": args.two_level, "build_s": build_s, "kmeans_iters": 5, "calls": rows}
 
+    # context for the HBM denominator: a pure read stream (torch sum-reduction over 4 GiB), since the
+    # measured copy peak mixes reads and writes
+    read_stream = None
+    if rank == 0:
+        try:
+            buf = torch.ones(1 << 29, dtype=torch.int64, device=dev)   # int64 sum: the fastest of torch's reductions here
+            for _ in range(2):
+                buf.sum()
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record()
+            for _ in range(5):
+                buf.sum()
+            ev1.record()
+            torch.cuda.synchronize()
+            read_stream = 5 * buf.numel() * 8 / (ev0.elapsed_time(ev1) * 1e-3) / 1e9
+            del buf
+        except RuntimeError:
+            read_stream = None
+
     clocks = sampler.stop() if sampler else None
 
     ms_all, q_all = aggregate_ranks(dist, main["ms"], float(nq * steps))
@@ -387,6 +406,7 @@ def run_ours(args):
                    "plan": plan, "l2": "slab is many times larger than L2 (126 MB): no flush between steps",
                    "replicas": world},
         "cache_entries_per_sec": mean_rows * nq * world / (ms_all / steps * 1e-3),
+        "read_stream_gb_per_sec": read_stream,
         "slab_gb_per_sec_whole_step": mean_rows * w.dim * 2 / (ms_all / steps * 1e-3) / 1e9,
         "gpu_launches": main["launches"],
         "e2e": e2e,

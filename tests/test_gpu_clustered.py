@@ -225,3 +225,10 @@ def test_index_lifecycle_and_errors():
         c.clear()
         assert c.index_info() == (0, 0)
         del before
+
+
+def test_more_queries_than_one_window():
+    # 1030 queries: two windows of the query loop, the second with six queries
+    w = _blob_workload(9_000, 64, 30, 0.3, seed=308, nq=1030)
+    x, q = wl.cache_rows(w, DEV), wl.queries(w, 1030, DEV)
+    _clustered_case(x, q, 6, 30, 2, 3, what="two-windows")
