@@ -59,6 +59,18 @@ def test_plan_paths_and_shapes():
     assert p["smem_bytes"] <= 232448
     assert p["seed_tiles"] > 0 and p["seed_tiles"] % 18 == 0 and p["seed_tiles"] * 256 * 15 < 16_000_000
     assert pkg.ic_cache_plan(768, 70_001, 64, 10)["seed_tiles"] == 0      # too few tiles per CTA
+    assert pkg.ic_cache_plan(768, 70_001, 64, 10)["seed0_tiles"] == 0
+    # threshold seeding: a maxima-only launch over about one tile per SM; a list-level sample of
+    # 1/16 of the tiles only on large caches; neither for a handful of queries with short lists
+    p = pkg.ic_cache_plan(768, 1_000_000, 64, 10)
+    assert (p["seed0_tiles"], p["seed_tiles"]) == (148, 0)
+    p = pkg.ic_cache_plan(768, 16_000_000, 64, 64)
+    assert p["seed0_tiles"] == 148 and p["seed_tiles"] == 16_000_000 // 256 // 16 // 148 * 148
+    p = pkg.ic_cache_plan(1024, 4_000_000, 256, 32)
+    assert p["seed0_tiles"] == 148 and p["seed_tiles"] % 74 == 0 and p["seed_tiles"] > 148
+    assert pkg.ic_cache_plan(768, 16_000_000, 1024, 64)["seed0_tiles"] == 162          # 9 tiles for each of 18 partitions
+    for nq, k, seeded in ((8, 10, False), (8, 16, False), (9, 10, True), (8, 17, True), (4, 64, True)):
+        assert (pkg.ic_cache_plan(768, 1_000_000, nq, k, path=pkg.IC_PATH_UMMA)["seed0_tiles"] > 0) == seeded
     p = pkg.ic_cache_plan(768, 16_000_000, 3000, 64)
     assert p["n_launches"] == 9
     assert pkg.ic_cache_plan(768, 1_000_000, 300, 10)["cta_group"] == 1    # odd number of query tiles
