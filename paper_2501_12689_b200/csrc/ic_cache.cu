@@ -416,10 +416,10 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
   // bf16 queries that need no normalisation go to the tensor-core path as they are: the query
   // tensor map points at the caller's rows and rows past nq read as zero, so the conversion
   // launch (and its place in the chain of dependent kernels) is saved.  Only with the last query
-  // tile at least half full: a tile that is mostly out-of-range rows loads slowly (measured:
-  // 16 queries, main pass 221 -> 261 us; 64 queries, step 282.5 -> 279.7 us).
+  // tile nearly full: out-of-range rows load slowly (measured main pass, 500-step runs: 64 queries
+  // 240 -> 262 us, 16 queries 221 -> 261 us; 100 and 128 queries unchanged, step 2-4 us shorter).
   const bool direct = pl.path == IC_PATH_UMMA && c->input_dtype == IC_BF16 && !c->normalize &&
-                      (reinterpret_cast<uintptr_t>(q) & 15) == 0 && nq_pad - nq <= QUERY_TILE / 2;
+                      (reinterpret_cast<uintptr_t>(q) & 15) == 0 && nq_pad - nq <= QUERY_TILE / 4;
   cudaError_t e = cudaSuccess;
   if (!direct) {
     e = icc::launch_convert_rows(q, c->input_dtype == IC_F32, nq, c->dim, c->normalize, c->q_bf16.p,
