@@ -199,6 +199,11 @@ def test_fp32_input_and_few_clusters():
 def test_index_lifecycle_and_errors():
     w = _blob_workload(4_000, 64, 10, 0.3, seed=307)
     x, q = wl.cache_rows(w, DEV), wl.queries(w, 3, DEV)
+    with ICCache(64, 8) as empty:
+        with pytest.raises(ICCacheError):
+            empty.build_index(0, 1)                              # nothing to cluster
+        assert empty.index_info() == (0, 0)
+        assert empty.utility_read()[0].numel() == 0
     with _cache_with(x, extra_capacity=16) as c:
         with pytest.raises(ICCacheError) as e:
             c.query_clustered(q, 4, 2)
@@ -217,6 +222,8 @@ def test_index_lifecycle_and_errors():
         with pytest.raises(ICCacheError):
             c.query_clustered(q, 4, 65)
         c.query_clustered(q, 4, 2)
+        none_ids, none_scores = c.query_clustered(q[:0], 4, 2)   # no queries: nothing to do
+        assert none_ids.shape == (0, 4) and none_scores.shape == (0, 4)
         before = c.query(q, 4)
         assert c.remove(wl.labels(1, "cpu")) == 1                # moving rows drops the index
         assert c.index_info() == (0, 0)
