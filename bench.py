@@ -3,7 +3,7 @@
 
 A step is one pass of the whole path over one query batch, as a serving loop would issue
 it: register the previous batch's requests (insert), then prepare, score, select and merge
-the new batch (query).  The default workload is the "online" configuration: 1,000,000 cached
+the new batch (query).  The clustered workload instead appends its 10,000 new rows per step.  The default workload is the "online" configuration: 1,000,000 cached
 bf16 embeddings of dimension 768, batch of 64 queries, k = 10.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload online] [--nq 64]
@@ -161,23 +161,36 @@ def barrier(dist):
     torch.cuda.synchronize()
 
 
-def timed_steps(cache, batches, ids_batches, k, steps, out_ids, out_scores, dist, first_step):
-    """K steps of [insert previous batch; query batch] timed with CUDA events on the stream
-    the library launches on (the current torch stream).  Returns (ms, wall window)."""
+def timed_steps(cache, batches, ins_batches, ids_batches, k, steps, out_ids, out_scores, dist, first_step,
+                time_inserts=False):
+    """K steps of [insert; query batch] timed with CUDA events on the stream the library launches
+    on (the current torch stream).  The inserted rows are the previous query batch (a served
+    request is registered afterwards) or, for a workload with streaming inserts, that step's own
+    batch of new rows (ins_batches).  Returns (ms, wall window, ms spent in the inserts or None)."""
     import torch
     nb = len(batches)
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    marks = []
     barrier(dist)
     w0 = time.time()
     start.record()
     for i in range(first_step, first_step + steps):
-        cache.insert(batches[(i - 1) % nb], ids_batches[i])
+        rows = ins_batches[i] if ins_batches is not None else batches[(i - 1) % nb]
+        if time_inserts:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            cache.insert(rows, ids_batches[i])
+            e1.record()
+            marks.append((e0, e1))
+        else:
+            cache.insert(rows, ids_batches[i])
         cache.query(batches[i % nb], k, out_ids, out_scores)
     stop.record()
     torch.cuda.synchronize()
     w1 = time.time()
     barrier(dist)
-    return start.elapsed_time(stop), (w0, w1)
+    ins_ms = sum(a.elapsed_time(b) for a, b in marks) if marks else None
+    return start.elapsed_time(stop), (w0, w1), ins_ms
 
 
 def run_ours(args):
@@ -191,15 +204,18 @@ def run_ours(args):
     if args.rows:
         w = w.scaled(args.rows)
     nq = args.nq or max(w.q_sweep)
-    steps = args.steps if args.steps is not None else 500
-    warmup = max(args.warmup if args.warmup is not None else 10, 3)
+    # a workload with streaming inserts appends insert_rows new rows per step: 20 steps by default
+    steps = args.steps if args.steps is not None else (20 if w.insert_rows else 500)
+    warmup = max(args.warmup if args.warmup is not None else (3 if w.insert_rows else 10), 3)
     path = {"auto": 0, "generic": 1, "scan": 2, "umma": 3}[args.path]
     peaks = load_peaks()
     props = torch.cuda.get_device_properties(dev)
 
     n_batches = 8
     max_nq = max(max(w.q_sweep), nq)
-    capacity = w.n + ((steps + warmup) * 4 + 64) * max_nq   # regions: value, profiled, e2e, sweeps
+    ins_rows = w.insert_rows if w.insert_rows else None      # rows appended per step (None: the previous batch)
+    per_step = max(max_nq, w.insert_rows)
+    capacity = w.n + ((steps + warmup) * (3 + len(w.q_sweep)) + 64) * per_step   # regions: value, profiled, e2e, sweeps
     cache = ICCache(w.dim, capacity, input_dtype=wl.torch_dtype(w))
     cache.set_path(path)
     x = wl.cache_rows(w, dev)
@@ -214,24 +230,29 @@ def run_ours(args):
         batches = [wl.queries(w, q, dev, round_idx=r) for r in range(n_batches)]
         first = step_counter[0] + 1
         tot = n_warm + n_steps
-        all_ids = wl.labels(tot * q, dev, first_slot=cache.size)   # labels follow slots
-        ids_batches = {first + j: all_ids[j * q:(j + 1) * q] for j in range(tot)}
+        ins = ins_rows or q
+        all_ids = wl.labels(tot * ins, dev, first_slot=cache.size)   # labels follow slots
+        ids_batches = {first + j: all_ids[j * ins:(j + 1) * ins] for j in range(tot)}
+        ins_batches = {first + j: wl.insert_batch(w, first + j, dev) for j in range(tot)} if ins_rows else None
         out_ids = torch.empty(q, w.k, dtype=torch.int64, device=dev)
         out_scores = torch.empty(q, w.k, dtype=torch.float32, device=dev)
-        timed_steps(cache, batches, ids_batches, w.k, n_warm, out_ids, out_scores, dist, first)
+        timed_steps(cache, batches, ins_batches, ids_batches, w.k, n_warm, out_ids, out_scores, dist, first)
         launches0 = cache.launch_count
         cache.set_profiling(profiled)
         if profiled:
             cache.read_profile()
         n_start = cache.size
-        ms, win = timed_steps(cache, batches, ids_batches, w.k, n_steps, out_ids, out_scores, dist, first + n_warm)
+        ms, win, ins_ms = timed_steps(cache, batches, ins_batches, ids_batches, w.k, n_steps, out_ids, out_scores, dist,
+                                      first + n_warm, time_inserts=profiled)
         prof = cache.read_profile() if profiled else None
+        if prof is not None:
+            prof["insert_ms"] = ins_ms
         cache.set_profiling(False)
         launches = cache.launch_count - launches0
         cache.sync()
         step_counter[0] += tot
-        # the cache grows by q rows per step: step j scans n_start + (j + 1) q rows
-        rows_scanned = n_steps * n_start + q * n_steps * (n_steps + 1) // 2
+        # the cache grows by `ins` rows per step: step j scans n_start + (j + 1) ins rows
+        rows_scanned = n_steps * n_start + ins * n_steps * (n_steps + 1) // 2
         if sampler:
             sampler.window(*win)
         return {"ms": ms, "steps": n_steps, "nq": q, "launches": launches, "profile": prof,
@@ -245,17 +266,24 @@ def run_ours(args):
     e2e_ms = None
     if not args.no_e2e:
         hb = [wl.queries(w, nq, dev, round_idx=r).cpu().pin_memory() for r in range(n_batches)]
-        h_ids = wl.labels((e2e_steps + warmup) * nq, "cpu", first_slot=cache.size).pin_memory()
+        ins = ins_rows or nq
+        h_ids = wl.labels((e2e_steps + warmup) * ins, "cpu", first_slot=cache.size).pin_memory()
+        # new rows of a streaming-insert workload: a few pinned batches, cycled
+        h_ins = [wl.insert_batch(w, 10_000 + r, dev).cpu().pin_memory() for r in range(4)] if ins_rows else None
         ho_ids = torch.empty(nq, w.k, dtype=torch.int64).pin_memory()
         ho_sc = torch.empty(nq, w.k, dtype=torch.float32).pin_memory()
+
+        def e2e_rows(i):
+            return h_ins[i % 4] if h_ins is not None else hb[(i - 1) % n_batches]
+
         for i in range(warmup):
-            cache.insert_host(hb[(i - 1) % n_batches], h_ids[i * nq:(i + 1) * nq])
+            cache.insert_host(e2e_rows(i), h_ids[i * ins:(i + 1) * ins])
             cache.query_host(hb[i % n_batches], w.k, ho_ids, ho_sc)
         barrier(dist)
         t0w = time.time()
         t0 = time.perf_counter()
         for i in range(warmup, warmup + e2e_steps):
-            cache.insert_host(hb[(i - 1) % n_batches], h_ids[i * nq:(i + 1) * nq])
+            cache.insert_host(e2e_rows(i), h_ids[i * ins:(i + 1) * ins])
             cache.query_host(hb[i % n_batches], w.k, ho_ids, ho_sc)
         torch.cuda.synchronize()
         e2e_ms = (time.perf_counter() - t0) * 1e3
@@ -263,7 +291,8 @@ def run_ours(args):
             sampler.window(t0w, time.time())
         barrier(dist)
     elem = 2 if w.input_dtype == "bf16" else 4
-    h2d = nq * w.dim * elem * 2 + nq * 8            # query batch + inserted rows + their ids
+    n_ins = ins_rows or nq
+    h2d = nq * w.dim * elem + n_ins * w.dim * elem + n_ins * 8   # query batch + inserted rows + their ids
     d2h = nq * w.k * 12
 
     sweep = []
@@ -387,6 +416,7 @@ def run_ours(args):
                     "launches_per_step": launches_per_step,
                     "algorithmic_bytes_per_launch": bytes_per_launch,
                     "rows_per_launch": rows_main,
+                    "insert_us_per_step": (pr["insert_ms"] * 1e3 / r["steps"]) if pr.get("insert_ms") is not None else None,
                     "seed_passes_us_per_step": pr["seed_ms"] * 1e3 / r["steps"],
                     "final_merge_us_per_step": pr["merge_ms"] * 1e3 / r["steps"]})
         return out
@@ -401,7 +431,8 @@ def run_ours(args):
         "ms_per_step": ms_all / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"{w.name}: N={w.n} d={w.dim} {w.input_dtype} unit {w.kind}, nq={nq}, k={w.k}",
-                   "step": "insert previous batch (nq rows) + query batch (prep, score, partial top-k, merge)",
+                   "step": (f"insert {w.insert_rows} new rows + query batch (prep, score, partial top-k, merge)" if w.insert_rows
+                            else "insert previous batch (nq rows) + query batch (prep, score, partial top-k, merge)"),
                    "n_start": main["n_start"], "n_end": main["n_end"], "path": binding.PATH_NAMES[plan["path"]],
                    "plan": plan, "l2": "slab is many times larger than L2 (126 MB): no flush between steps",
                    "replicas": world},
