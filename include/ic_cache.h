@@ -53,7 +53,7 @@ enum ic_dtype { IC_BF16 = 0, IC_F32 = 1 };
 
 /* Kernel path used for scoring (see ic_cache_plan). */
 enum ic_path {
-  IC_PATH_AUTO = 0,    /* scan for one or two queries (dim <= 1024), tensor cores otherwise */
+  IC_PATH_AUTO = 0,    /* scan for one or two queries (512 <= dim <= 1024), tensor cores otherwise */
   IC_PATH_GENERIC = 1, /* plain CUDA-core kernel, any shape; slow, kept as a cross-check  */
   IC_PATH_SCAN = 2,    /* bulk-copy staged CUDA-core scan, nq <= 4 per pass, dim <= 1024  */
   IC_PATH_UMMA = 3     /* tcgen05 tensor-core tiles with the top-k fused in the epilogue  */

@@ -37,6 +37,7 @@ constexpr int UMMA_STAGE_BYTES = (QUERY_TILE + ROW_TILE) * K_CHUNK * 2;  // 48 K
 constexpr int SCAN_MAX_Q = 4;        // queries per scan launch
 constexpr int SCAN_AUTO_MAX_Q = 2;   // largest batch the automatic choice gives to the scan path
 constexpr int SCAN_MAX_DIM = 1024;
+constexpr int SCAN_AUTO_MIN_DIM = 512;   // shorter rows go to the tensor-core path even for one query
 constexpr int SCAN_ROWS_PER_STAGE = 32;
 constexpr int SCAN_CONSUMER_WARPS = 8;
 constexpr int GENERIC_QB = 4;
@@ -172,7 +173,10 @@ int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32
   const int n_windows = (nq + WINDOW_MAX_NQ - 1) / WINDOW_MAX_NQ;
   // measured crossover (N = 1 M, d = 768, k = 10): the scan wins for one or two queries, the
   // tensor-core path from three on (its time hardly grows with nq while HBM-bound)
-  if (path == IC_PATH_AUTO) path = (nq <= SCAN_AUTO_MAX_Q && dim <= SCAN_MAX_DIM) ? IC_PATH_SCAN : IC_PATH_UMMA;
+  // (and only for rows of at least 1 KiB: at dim = 384, N = 2 M, one query takes 271 us on the scan
+  // against 245 us on the tensor-core path; at dim = 768 and 1024 the scan is 2-4 % ahead in long runs)
+  if (path == IC_PATH_AUTO)
+    path = (nq <= SCAN_AUTO_MAX_Q && dim <= SCAN_MAX_DIM && dim >= SCAN_AUTO_MIN_DIM) ? IC_PATH_SCAN : IC_PATH_UMMA;
   out->path = path;
   const int merge_lists_max = (smem_optin - 4096) / (k * 8 + 4);
   if (path == IC_PATH_GENERIC) {
