@@ -377,3 +377,48 @@ def test_expired_device_wait_is_reported_and_the_handle_recovers():
         after = c.query(q, 4)
         c.sync()
         assert torch.equal(before[0], after[0]) and torch.equal(before[1], after[1])
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_random_shapes_tensor_core_path_agrees_with_the_plain_kernel(seed):
+    """Seeded random shapes, large enough to reach the seeding launches and CTA pairs, where the
+    oracle would take too long: the tensor-core path and the automatic choice must agree with the
+    plain CUDA-core kernel (itself checked against the oracle above) up to ties at the k-th place."""
+    import random
+    rng = random.Random(seed)
+    for case in range(12):
+        dim = rng.choice([8, 64, 128, 384, 520, 768, 1024, 1536])
+        n = rng.choice([rng.randint(1, 3000), rng.randint(3000, 80_000), rng.randint(80_000, 700_000)])
+        n = min(n, 400_000_000 // dim)
+        nq = rng.choice([1, 2, 3, 7, 9, 33, 64, 65, 128, 129, 257])
+        k = rng.choice([1, 2, 8, 10, 16, 17, 32, 64, 100, 128])
+        kind = rng.choice(["gaussian", "clustered", "sorted"])
+        w = wl.Workload("f", n, dim, "bf16", (nq,), k, seed=7000 + 100 * seed + case,
+                        kind="clustered" if kind == "clustered" else "gaussian", n_clusters=50, sigma=0.3,
+                        dup_frac=0.01 if kind == "clustered" else 0.0)
+        x, q = wl.cache_rows(w, DEV), wl.queries(w, nq, DEV)
+        if kind == "sorted":
+            x = x[torch.argsort(x.float() @ q[0].float(), descending=rng.random() < 0.5)].contiguous()
+        got = {}
+        with ICCache(dim, n) as c:
+            c.insert(x, wl.labels(n, DEV))
+            for name, path in (("umma", IC_PATH_UMMA), ("auto", IC_PATH_AUTO), ("plain", IC_PATH_GENERIC)):
+                c.set_path(path)
+                ids, sc = c.query(q, k)
+                c.sync()
+                got[name] = (ids.cpu(), sc.cpu())
+        p_ids, p_sc = got["plain"]
+        fin = torch.isfinite(p_sc)
+        what = f"seed {seed} case {case}: dim {dim} n {n} nq {nq} k {k} {kind}"
+        for name in ("umma", "auto"):
+            a_ids, a_sc = got[name]
+            assert torch.equal(torch.isfinite(a_sc), fin), what
+            if fin.any():
+                assert (a_sc[fin] - p_sc[fin]).abs().max().item() <= 1e-4, what
+            for i in range(nq):
+                sa, sp = set(a_ids[i].tolist()), set(p_ids[i].tolist())
+                if sa != sp:     # only entries tied with the k-th score may differ
+                    kth = p_sc[i][fin[i]].min().item()
+                    for arr_ids, arr_sc in ((a_ids[i], a_sc[i]), (p_ids[i], p_sc[i])):
+                        for j, idv in enumerate(arr_ids.tolist()):
+                            assert idv not in (sa ^ sp) or abs(arr_sc[j].item() - kth) <= 2e-4, what
