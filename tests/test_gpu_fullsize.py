@@ -135,3 +135,18 @@ def test_two_level_search_at_full_size(loaded):
     e, g = exact_ids.cpu().numpy(), ids.cpu().numpy()
     recall = np.mean([len(set(e[i]) & set(g[i])) / w.k for i in range(nq)])
     assert recall > 0.95, recall
+
+
+@pytest.mark.parametrize("name,rows", [("dense", 160_003), ("stress", 70_000)])
+def test_every_query_of_the_large_batches_on_a_truncated_cache(name, rows):
+    """The full-size checks above sample a few queries per batch.  Here every query of the two
+    large-batch workloads (256 and 1024 queries: two and eight query tiles, CTA pairs, seeding)
+    is checked against the oracle, on a cache cut down to 160,003 / 70,000 rows of the same
+    recipe (still enough tiles per CTA for the seeding launch) so that the oracle finishes soon."""
+    from parity_util import run_and_check
+    w = wl.WORKLOADS[name].scaled(rows)
+    nq = max(w.q_sweep)
+    plan = ic_cache_plan(w.dim, w.n, nq, w.k, IC_PATH_AUTO)
+    assert plan["n_query_tiles"] == nq // 128 and plan["cta_group"] == 2 and plan["seed0_tiles"] > 0
+    x, q = wl.cache_rows(w, DEV), wl.queries(w, nq, DEV)
+    run_and_check(x, q, w.k, path=IC_PATH_AUTO, what=f"{name}/truncated/all-queries")
