@@ -72,6 +72,10 @@ typedef struct ic_cache_opts {
                            256-byte aligned; NULL = the library allocates                  */
   void* ids;            /* optional caller-owned device buffer, capacity*8 bytes           */
   void* stream;         /* cudaStream_t; NULL = the legacy default stream                  */
+  void* workspace;      /* optional caller-owned device buffer (256-byte aligned) that serves
+                           as the scratch of ic_cache_query / ic_cache_query_min_score, which
+                           then allocate nothing; NULL = the library grows its own buffers   */
+  size_t workspace_bytes; /* its size; see ic_cache_workspace_bytes                          */
 } ic_cache_opts_t;
 
 /* Host-side launch plan for one query call; pure function of its arguments. */
@@ -130,6 +134,18 @@ int ic_cache_insert(ic_cache_t* c, const void* emb, const int64_t* ids, int64_t 
  */
 int ic_cache_query(ic_cache_t* c, const void* q, int32_t nq, int32_t k, int64_t* out_ids,
                    float* out_scores);
+
+/*
+ * Bytes of workspace (ic_cache_opts_t.workspace) that ic_cache_query needs at most for batches
+ * of up to max_nq queries and k up to max_k against up to `capacity` entries of dimension dim,
+ * on the current CUDA device (the launch plan depends on its SM count; without a device the
+ * figures of a B200 are used).  0 for invalid arguments.  With a workspace the handle's
+ * queries take all scratch (query staging, partial lists, floors, group maxima) from it and
+ * return IC_ERR_NOMEM, enqueuing nothing, when a call needs more than it holds; the other
+ * calls (host variants, self-similarity, index, removal) still use library-owned buffers.  Like
+ * the static scratch, a workspace must not be shared by calls that overlap on the GPU.
+ */
+size_t ic_cache_workspace_bytes(int32_t dim, int64_t capacity, int32_t max_nq, int32_t max_k);
 
 /*
  * ic_cache_query that reports only entries whose score reaches min_score: the hit test of

@@ -35,6 +35,8 @@ class ic_cache_opts_t(ctypes.Structure):
         ("slab", ctypes.c_void_p),
         ("ids", ctypes.c_void_p),
         ("stream", ctypes.c_void_p),
+        ("workspace", ctypes.c_void_p),
+        ("workspace_bytes", ctypes.c_size_t),
     ]
 
 
@@ -62,6 +64,7 @@ SIGNATURES = {
     "ic_cache_insert": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64]),
     "ic_cache_query": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
                                       ctypes.c_void_p, ctypes.c_void_p]),
+    "ic_cache_workspace_bytes": (ctypes.c_size_t, [ctypes.c_int32, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32]),
     "ic_cache_query_min_score": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
                                                 ctypes.c_float, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "ic_cache_query_static": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
@@ -139,7 +142,8 @@ def ic_cache_create(dim: int, capacity: int):
 
 def ic_cache_create_ex(dim: int, capacity: int, *, device: int = -1, input_dtype: int = IC_BF16,
                        normalize: bool = False, slab: Optional[torch.Tensor] = None,
-                       ids: Optional[torch.Tensor] = None, stream: int = 0):
+                       ids: Optional[torch.Tensor] = None, stream: int = 0,
+                       workspace: Optional[torch.Tensor] = None):
     o = ic_cache_opts_t()
     o.struct_size = ctypes.sizeof(ic_cache_opts_t)
     o.device = device
@@ -148,10 +152,16 @@ def ic_cache_create_ex(dim: int, capacity: int, *, device: int = -1, input_dtype
     o.slab = slab.data_ptr() if slab is not None else None
     o.ids = ids.data_ptr() if ids is not None else None
     o.stream = stream or None
+    o.workspace = workspace.data_ptr() if workspace is not None else None
+    o.workspace_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
     h = load_library().ic_cache_create_ex(dim, capacity, ctypes.byref(o))
     if not h:
         raise ICCacheError(IC_ERR_INVALID, ic_cache_last_error())
     return h
+
+
+def ic_cache_workspace_bytes(dim: int, capacity: int, max_nq: int, max_k: int) -> int:
+    return int(load_library().ic_cache_workspace_bytes(dim, capacity, max_nq, max_k))
 
 
 def ic_cache_insert(h, emb: torch.Tensor, ids: torch.Tensor, n: Optional[int] = None) -> None:
@@ -201,7 +211,8 @@ class ICCache:
     chosen at construction."""
 
     def __init__(self, dim: int, capacity: int, *, input_dtype: torch.dtype = torch.bfloat16,
-                 normalize: bool = False, device: Optional[int] = None, stream: Optional[torch.cuda.Stream] = None):
+                 normalize: bool = False, device: Optional[int] = None, stream: Optional[torch.cuda.Stream] = None,
+                 workspace: Optional[torch.Tensor] = None):
         if input_dtype not in (torch.bfloat16, torch.float32):
             raise TypeError("input_dtype must be torch.bfloat16 or torch.float32")
         self.dim, self.capacity, self.input_dtype = dim, capacity, input_dtype
@@ -210,7 +221,8 @@ class ICCache:
         st = stream if stream is not None else torch.cuda.current_stream(self.device)
         self._h = ic_cache_create_ex(
             dim, capacity, device=dev, input_dtype=IC_F32 if input_dtype == torch.float32 else IC_BF16,
-            normalize=normalize, stream=st.cuda_stream)
+            normalize=normalize, stream=st.cuda_stream, workspace=workspace)
+        self._workspace = workspace     # borrowed by the handle: keep it alive
 
     # -- lifetime
     def close(self) -> None:

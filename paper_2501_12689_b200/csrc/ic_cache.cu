@@ -95,6 +95,8 @@ struct ic_cache {
   ic_cache* centroids = nullptr;
   int32_t n_clusters = 0;
   int64_t n_indexed = 0;
+  unsigned char* workspace = nullptr;   // optional caller-owned scratch for ic_cache_query (borrowed)
+  size_t workspace_bytes = 0;
   float* utility = nullptr;   // [capacity] per-entry utility, allocated on first use, zero for new entries
   Buffer util_ids, util_gains;
   Buffer idx_assign, idx_best, idx_order, idx_offsets, idx_sort, idx_init, idx_probes, idx_probe_scores;
@@ -505,35 +507,47 @@ int static_scratch_address(int dev, unsigned char** out) {
   return IC_OK;
 }
 
-// One query window with all scratch taken from the static array.  Mirrors do_query_window
-// but never grows a buffer, creates an event or allocates in any other way.
-int do_query_window_static(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids, float* out_scores) {
-  const float min_score = -INFINITY;
-  int32_t* const out_counts = nullptr;
+// Where the pieces of a query window's scratch sit inside one fixed block (the static array or a
+// caller's workspace), and how much of it the window needs.
+struct FixedLayout {
+  size_t off_qbf16, off_qf32, off_part, off_thr, off_max, off_pace, need;
+};
+
+FixedLayout fixed_layout(int dim, int nq, int k, const ic_cache_plan_t& pl) {
+  const int nq_pad = (nq + QUERY_TILE - 1) / QUERY_TILE * QUERY_TILE;
+  const size_t list_block = (size_t)nq * k;
+  auto round_up = [](size_t v) { return (v + 1023) & ~(size_t)1023; };
+  FixedLayout f;
+  f.off_qbf16 = 0;
+  f.off_qf32 = f.off_qbf16 + round_up((size_t)nq_pad * dim * 2);
+  f.off_part = f.off_qf32 + round_up((size_t)nq * dim * 4);
+  f.off_thr = f.off_part + round_up((size_t)(2 * pl.n_partitions + 2) * list_block * 8);
+  f.off_max = f.off_thr + round_up((size_t)nq * 8);
+  f.off_pace = f.off_max + round_up((size_t)pl.seed0_tiles * nq * 16);
+  f.need = f.off_pace + PACE_BYTES;
+  return f;
+}
+
+// One query window with all scratch taken from a fixed block of `block_bytes` at `base` (NULL: the
+// static array of this device).  Mirrors do_query_window but never grows a buffer, creates an
+// event or allocates in any other way.
+int do_query_window_fixed(ic_cache* c, unsigned char* base, size_t block_bytes, const char* block_name, const void* q,
+                          int nq, int k, int64_t* out_ids, float* out_scores, float min_score, int32_t* out_counts) {
   ic_cache_plan_t pl;
   int rc = plan_impl(c->dim, c->size, nq, k, c->forced_path, c->sm_count, c->smem_optin, &pl);
   if (rc != IC_OK) return rc;
   const int nq_pad = (nq + QUERY_TILE - 1) / QUERY_TILE * QUERY_TILE;
-  const size_t list_block = (size_t)nq * k;
-  auto round_up = [](size_t v) { return (v + 1023) & ~(size_t)1023; };
-  const size_t off_qbf16 = 0;
-  const size_t off_qf32 = off_qbf16 + round_up((size_t)nq_pad * c->dim * 2);
-  const size_t off_part = off_qf32 + round_up((size_t)nq * c->dim * 4);
-  const size_t off_thr = off_part + round_up((size_t)(2 * pl.n_partitions + 2) * list_block * 8);
-  const size_t off_max = off_thr + round_up((size_t)nq * 8);
-  const size_t off_pace = off_max + round_up((size_t)pl.seed0_tiles * nq * 16);
-  const size_t need = off_pace + PACE_BYTES;
-  if (need > (size_t)IC_STATIC_SCRATCH_BYTES)
-    return fail(IC_ERR_NOMEM, "query needs %zu bytes of scratch but the static scratch holds %u; use ic_cache_query or a smaller nq/k",
-                need, (unsigned)IC_STATIC_SCRATCH_BYTES);
-  unsigned char* base = nullptr;
-  if ((rc = static_scratch_address(c->device, &base)) != IC_OK) return rc;
-  void* q_bf16 = base + off_qbf16;
-  float* q_f32 = reinterpret_cast<float*>(base + off_qf32);
-  uint64_t* partials = reinterpret_cast<uint64_t*>(base + off_part);
-  uint64_t* thr = reinterpret_cast<uint64_t*>(base + off_thr);
-  float* maxima = reinterpret_cast<float*>(base + off_max);
-  unsigned long long* pace = reinterpret_cast<unsigned long long*>(base + off_pace);
+  const FixedLayout f = fixed_layout(c->dim, nq, k, pl);
+  if (f.need > block_bytes)
+    return fail(IC_ERR_NOMEM, "query needs %zu bytes of scratch but the %s holds %zu; use a smaller nq/k or a handle without it",
+                f.need, block_name, block_bytes);
+  if (!base && (rc = static_scratch_address(c->device, &base)) != IC_OK) return rc;
+  void* q_bf16 = base + f.off_qbf16;
+  float* q_f32 = reinterpret_cast<float*>(base + f.off_qf32);
+  uint64_t* partials = reinterpret_cast<uint64_t*>(base + f.off_part);
+  uint64_t* thr = reinterpret_cast<uint64_t*>(base + f.off_thr);
+  float* maxima = reinterpret_cast<float*>(base + f.off_max);
+  unsigned long long* pace = reinterpret_cast<unsigned long long*>(base + f.off_pace);
 
   cudaError_t e = icc::launch_convert_rows(q, c->input_dtype == IC_F32, nq, c->dim, c->normalize, q_bf16, q_f32, nq_pad,
                                            nullptr, nullptr, c->stream);
@@ -707,6 +721,8 @@ ic_cache_t* ic_cache_create_ex(int32_t dim, int64_t capacity, const ic_cache_opt
   c->input_dtype = o.input_dtype;
   c->normalize = o.normalize ? 1 : 0;
   c->stream = static_cast<cudaStream_t>(o.stream);
+  c->workspace = static_cast<unsigned char*>(o.workspace);
+  c->workspace_bytes = o.workspace ? o.workspace_bytes : 0;
   c->sm_count = prop.multiProcessorCount;
   c->smem_optin = (int)prop.sharedMemPerBlockOptin;
   c->l2_bytes = prop.l2CacheSize;
@@ -727,6 +743,12 @@ ic_cache_t* ic_cache_create_ex(int32_t dim, int64_t capacity, const ic_cache_opt
       ok = false;
     }
     c->own_slab = ok;
+  }
+  if (ok && o.workspace) {
+    if (!is_device_ptr(o.workspace, dev) || (reinterpret_cast<uintptr_t>(o.workspace) & 255)) {
+      fail(IC_ERR_INVALID, "opts.workspace must be a 256-byte aligned device pointer on device %d", dev);
+      ok = false;
+    }
   }
   if (ok) {
     if (o.ids) {
@@ -917,11 +939,47 @@ int ic_cache_query_min_score(ic_cache_t* c, const void* q, int32_t nq, int32_t k
   const size_t q_row = (size_t)c->dim * in_elem_bytes(c);
   for (int q0 = 0; q0 < nq; q0 += WINDOW_MAX_NQ) {
     const int w = std::min(WINDOW_MAX_NQ, nq - q0);
-    rc = do_query_window(c, static_cast<const char*>(q) + (size_t)q0 * q_row, w, k, out_ids + (size_t)q0 * k,
-                         out_scores + (size_t)q0 * k, min_score, out_counts ? out_counts + q0 : nullptr);
+    const char* qw = static_cast<const char*>(q) + (size_t)q0 * q_row;
+    if (c->workspace)   // caller-owned scratch: nothing is allocated, too small a workspace is an error
+      rc = do_query_window_fixed(c, c->workspace, c->workspace_bytes, "caller's workspace", qw, w, k,
+                                 out_ids + (size_t)q0 * k, out_scores + (size_t)q0 * k, min_score,
+                                 out_counts ? out_counts + q0 : nullptr);
+    else
+      rc = do_query_window(c, qw, w, k, out_ids + (size_t)q0 * k, out_scores + (size_t)q0 * k, min_score,
+                           out_counts ? out_counts + q0 : nullptr);
     if (rc != IC_OK) return rc;
   }
   return IC_OK;
+}
+
+size_t ic_cache_workspace_bytes(int32_t dim, int64_t capacity, int32_t max_nq, int32_t max_k) {
+  if (dim < 8 || dim > IC_MAX_DIM || (dim % 8) != 0 || capacity < 1 || max_nq < 1 || max_k < 1 || max_k > IC_MAX_K) {
+    fail(IC_ERR_INVALID, "workspace_bytes: bad dim, capacity, max_nq or max_k");
+    return 0;
+  }
+  // the launch plan depends on the device: the current one when there is one, else a B200's figures
+  int sm_count = 148, smem_optin = 232448, dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) == cudaSuccess && cudaGetDeviceProperties(&prop, dev) == cudaSuccess) {
+    sm_count = prop.multiProcessorCount;
+    smem_optin = (int)prop.sharedMemPerBlockOptin;
+  } else {
+    cudaGetLastError();
+  }
+  // a call is served in windows of at most 1024 queries; within a given number of query tiles the
+  // need grows with nq, so the largest batch of every tile count (and one or two queries, which
+  // may take the scan path) covers all shapes
+  const int limit = std::min<int>(max_nq, WINDOW_MAX_NQ);
+  size_t need = 0;
+  for (int cand = 0; cand <= WINDOW_MAX_NQ / QUERY_TILE + 1; ++cand) {
+    const int nq = cand == 0 ? 1 : (cand == 1 ? std::min(2, limit) : std::min((cand - 1) * QUERY_TILE, limit));
+    for (int path : {(int)IC_PATH_AUTO, (int)IC_PATH_UMMA}) {
+      ic_cache_plan_t pl;
+      if (plan_impl(dim, capacity, nq, max_k, path, sm_count, smem_optin, &pl) != IC_OK) continue;
+      need = std::max(need, fixed_layout(dim, nq, max_k, pl).need);
+    }
+  }
+  return need;
 }
 
 int ic_cache_query_static(ic_cache_t* c, const void* q, int32_t nq, int32_t k, int64_t* out_ids, float* out_scores) {
@@ -932,7 +990,8 @@ int ic_cache_query_static(ic_cache_t* c, const void* q, int32_t nq, int32_t k, i
   if (!is_device_ptr(q, c->device) || !is_device_ptr(out_ids, c->device) || !is_device_ptr(out_scores, c->device))
     return fail(IC_ERR_INVALID, "q, out_ids and out_scores must be device pointers on device %d", c->device);
   if ((rc = check_timeout(c)) != IC_OK) return rc;
-  return do_query_window_static(c, q, nq, k, out_ids, out_scores);
+  return do_query_window_fixed(c, nullptr, IC_STATIC_SCRATCH_BYTES, "static scratch", q, nq, k, out_ids, out_scores,
+                               -INFINITY, nullptr);
 }
 
 int ic_cache_query_host(ic_cache_t* c, const void* q_host, int32_t nq, int32_t k, int64_t* out_ids_host,

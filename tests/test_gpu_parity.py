@@ -422,3 +422,38 @@ def test_random_shapes_tensor_core_path_agrees_with_the_plain_kernel(seed):
                     for arr_ids, arr_sc in ((a_ids[i], a_sc[i]), (p_ids[i], p_sc[i])):
                         for j, idv in enumerate(arr_ids.tolist()):
                             assert idv not in (sa ^ sp) or abs(arr_sc[j].item() - kth) <= 2e-4, what
+
+
+def test_caller_owned_workspace_serves_queries_without_allocation():
+    """A handle created with a workspace of ic_cache_workspace_bytes takes the scratch of its
+    queries from it: same results as a handle that grows its own buffers, for every kernel path
+    the automatic choice reaches; a workspace that is too small is an error, not an allocation."""
+    from paper_2501_12689_b200 import ic_cache_workspace_bytes, IC_ERR_NOMEM
+    w = wl.WORKLOADS["online"].scaled(400_003)         # enough tiles for the seeding launches
+    x = wl.cache_rows(w, DEV)
+    ids = wl.labels(w.n, DEV)
+    need = ic_cache_workspace_bytes(w.dim, w.n, 300, 16)
+    ws = torch.empty(need, dtype=torch.uint8, device=DEV)
+    with ICCache(w.dim, w.n) as plain, ICCache(w.dim, w.n, workspace=ws) as fixed:
+        plain.insert(x, ids)
+        fixed.insert(x, ids)
+        for nq, k in ((1, 10), (2, 16), (5, 3), (64, 10), (130, 16), (300, 8)):
+            q = wl.queries(w, nq, DEV, round_idx=nq)
+            a_ids, a_sc = plain.query(q, k)
+            b_ids, b_sc = fixed.query(q, k)
+            plain.sync()
+            fixed.sync()
+            assert torch.equal(a_ids, b_ids) and torch.equal(a_sc, b_sc), f"nq {nq} k {k}"
+        c_ids, c_sc, c_cnt = fixed.query_min_score(wl.queries(w, 7, DEV), 5, 0.12)
+        d_ids, d_sc, d_cnt = plain.query_min_score(wl.queries(w, 7, DEV), 5, 0.12)
+        assert torch.equal(c_ids, d_ids) and torch.equal(c_cnt, d_cnt)
+        with pytest.raises(ICCacheError) as e:                 # beyond what the workspace was sized for
+            fixed.query(wl.queries(w, 1024, DEV), 64)
+        assert e.value.status == IC_ERR_NOMEM
+        fixed.query(wl.queries(w, 3, DEV), 4)                  # the handle stays usable
+    tiny = torch.empty(4096, dtype=torch.uint8, device=DEV)
+    with ICCache(w.dim, 1000, workspace=tiny) as c:
+        c.insert(x[:1000], ids[:1000])
+        with pytest.raises(ICCacheError) as e:
+            c.query(wl.queries(w, 1, DEV), 1)
+        assert e.value.status == IC_ERR_NOMEM

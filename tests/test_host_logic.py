@@ -82,6 +82,20 @@ def test_plan_paths_and_shapes():
         assert pkg.ic_cache_plan(4096, 10, 128, k)["n_stages"] >= 2
 
 
+def test_workspace_bytes_covers_every_batch_shape_up_to_the_limits():
+    # pure host arithmetic (B200 figures without a device): enough for the largest batch of every
+    # query-tile count, growing with the limits, zero for bad arguments
+    small = pkg.ic_cache_workspace_bytes(768, 1_000_000, 64, 10)
+    big = pkg.ic_cache_workspace_bytes(768, 1_000_000, 1024, 64)
+    assert 0 < small < big < (1 << 30)
+    assert pkg.ic_cache_workspace_bytes(768, 1_000_000, 5000, 64) == big       # windows of 1024 queries
+    assert pkg.ic_cache_workspace_bytes(768, 16_000_000, 64, 10) >= small      # more seeding tiles at most
+    # query staging alone: bf16 padded to 128 rows plus fp32
+    assert small >= 128 * 768 * 2 + 64 * 768 * 4
+    for bad in [(12, 10, 1, 1), (768, 0, 1, 1), (768, 10, 0, 1), (768, 10, 1, 0), (768, 10, 1, 129)]:
+        assert pkg.ic_cache_workspace_bytes(*bad) == 0
+
+
 @pytest.mark.parametrize("args", [
     dict(dim=12, n=10, nq=1, k=1), dict(dim=0, n=10, nq=1, k=1), dict(dim=8192, n=10, nq=1, k=1),
     dict(dim=64, n=10, nq=0, k=1), dict(dim=64, n=10, nq=1, k=0), dict(dim=64, n=10, nq=1, k=129),
