@@ -235,6 +235,19 @@ int ic_cache_self_similarity(ic_cache_t* c, int64_t first, int64_t count, int64_
 int ic_cache_remove(ic_cache_t* c, const int64_t* ids_host, int64_t n, int64_t* n_removed);
 
 /*
+ * Checkpoint and restore (paper Sec. 5, "Fault Tolerance": every component periodically
+ * checkpoints its state).  ic_cache_save writes the entries (stored bf16 rows, ids, utilities if
+ * any) to a file on the HOST file system; ic_cache_load replaces the handle's contents with a
+ * file written by ic_cache_save for the same dimension (size at most this handle's capacity),
+ * keeping slots, ids and utilities, so queries return exactly what they returned before.  Both
+ * synchronise the stream and copy through host memory; neither is part of the per-request path.
+ * The two-level index is not stored: rebuild it after loading.  On a failed load the handle is
+ * left empty.  IC_ERR_INVALID for an unreadable, foreign or mismatching file.
+ */
+int ic_cache_save(ic_cache_t* c, const char* path);
+int ic_cache_load(ic_cache_t* c, const char* path);
+
+/*
  * Per-entry utility for the cache-management policy (paper Sec. 4.3, "Example Manager": each
  * example's value is the efficiency gain it enabled, i.e. the number of successful offloadings,
  * kept as a moving average that is multiplied by 0.9 every hour; a knapsack solver run by the

@@ -75,6 +75,8 @@ SIGNATURES = {
     "ic_cache_self_similarity": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
                                                 ctypes.c_void_p]),
     "ic_cache_remove": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.POINTER(ctypes.c_int64)]),
+    "ic_cache_save": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_char_p]),
+    "ic_cache_load": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_char_p]),
     "ic_cache_utility_add": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64]),
     "ic_cache_utility_decay": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_float]),
     "ic_cache_utility_read": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
@@ -314,6 +316,14 @@ class ICCache:
         out_scores = torch.empty(count, dtype=torch.float32, device=self.device)
         _check(load_library().ic_cache_self_similarity(self._h, first, count, _ptr(out_ids), _ptr(out_scores)))
         return out_ids, out_scores
+
+    def save(self, path: str) -> None:
+        """Write the entries (rows, ids, utilities) to a checkpoint file."""
+        _check(load_library().ic_cache_save(self._h, os.fsencode(path)))
+
+    def load(self, path: str) -> None:
+        """Replace the contents with a checkpoint written by save() for the same dimension."""
+        _check(load_library().ic_cache_load(self._h, os.fsencode(path)))
 
     def utility_add(self, ids: torch.Tensor, gains: torch.Tensor) -> None:
         """Add gains[i] to the utility of every entry whose id is ids[i] (host int64 / float32 tensors)."""

@@ -1105,6 +1105,95 @@ int ic_cache_self_similarity(ic_cache_t* c, int64_t first, int64_t count, int64_
   return query_bf16_rows(c, q_rows, count, c->capacity - first, k, out_ids, out_scores, first);
 }
 
+// ------------------------------------------------------------------ checkpoint file
+// Layout: a 64-byte header, then size*dim bf16 rows, size int64 ids, and (flag) size fp32 utilities.
+namespace {
+struct CheckpointHeader {
+  char magic[8];        // "ICCKPT01"
+  int32_t dim;
+  int32_t has_utility;
+  int64_t size;
+  int64_t reserved[5];
+};
+static_assert(sizeof(CheckpointHeader) == 64, "checkpoint header is 64 bytes");
+constexpr size_t CKPT_CHUNK = (size_t)32 << 20;
+
+// Stream `bytes` between a device range and the file through a host bounce buffer.
+int copy_device_file(void* dev, size_t bytes, FILE* f, bool to_file, std::vector<unsigned char>& bounce, const char* path) {
+  for (size_t off = 0; off < bytes; off += CKPT_CHUNK) {
+    const size_t len = std::min(CKPT_CHUNK, bytes - off);
+    if (to_file) {
+      if (cudaMemcpy(bounce.data(), static_cast<char*>(dev) + off, len, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return fail(IC_ERR_CUDA, "device-to-host copy failed while writing %s", path);
+      if (fwrite(bounce.data(), 1, len, f) != len) return fail(IC_ERR_INVALID, "short write to %s", path);
+    } else {
+      if (fread(bounce.data(), 1, len, f) != len) return fail(IC_ERR_INVALID, "%s is truncated", path);
+      if (cudaMemcpy(static_cast<char*>(dev) + off, bounce.data(), len, cudaMemcpyHostToDevice) != cudaSuccess)
+        return fail(IC_ERR_CUDA, "host-to-device copy failed while reading %s", path);
+    }
+  }
+  return IC_OK;
+}
+}  // namespace
+
+int ic_cache_save(ic_cache_t* c, const char* path) {
+  if (!c || !path) return fail(IC_ERR_INVALID, "NULL handle or path");
+  DeviceGuard guard(c->device);
+  int rc = ic_cache_sync(c);
+  if (rc != IC_OK) return rc;
+  FILE* f = fopen(path, "wb");
+  if (!f) return fail(IC_ERR_INVALID, "cannot open %s for writing", path);
+  CheckpointHeader h;
+  memset(&h, 0, sizeof h);
+  memcpy(h.magic, "ICCKPT01", 8);
+  h.dim = c->dim;
+  h.has_utility = c->utility ? 1 : 0;
+  h.size = c->size;
+  std::vector<unsigned char> bounce(std::min(CKPT_CHUNK, std::max<size_t>(1, (size_t)c->size * c->dim * 2)));
+  rc = fwrite(&h, sizeof h, 1, f) == 1 ? IC_OK : fail(IC_ERR_INVALID, "short write to %s", path);
+  if (rc == IC_OK) rc = copy_device_file(c->slab, (size_t)c->size * c->dim * 2, f, true, bounce, path);
+  if (rc == IC_OK) rc = copy_device_file(c->ids, (size_t)c->size * 8, f, true, bounce, path);
+  if (rc == IC_OK && c->utility) rc = copy_device_file(c->utility, (size_t)c->size * 4, f, true, bounce, path);
+  if (fclose(f) != 0 && rc == IC_OK) rc = fail(IC_ERR_INVALID, "closing %s failed", path);
+  return rc;
+}
+
+int ic_cache_load(ic_cache_t* c, const char* path) {
+  if (!c || !path) return fail(IC_ERR_INVALID, "NULL handle or path");
+  DeviceGuard guard(c->device);
+  int rc = ic_cache_sync(c);
+  if (rc != IC_OK) return rc;
+  FILE* f = fopen(path, "rb");
+  if (!f) return fail(IC_ERR_INVALID, "cannot open %s", path);
+  CheckpointHeader h;
+  if (fread(&h, sizeof h, 1, f) != 1 || memcmp(h.magic, "ICCKPT01", 8) != 0) {
+    fclose(f);
+    return fail(IC_ERR_INVALID, "%s is not a cache checkpoint", path);
+  }
+  if (h.dim != c->dim || h.size < 0 || h.size > c->capacity) {
+    fclose(f);
+    return fail(IC_ERR_INVALID, "%s holds %lld entries of dimension %d; this handle has dimension %d and capacity %lld",
+                path, (long long)h.size, h.dim, c->dim, (long long)c->capacity);
+  }
+  if (h.has_utility && (rc = ensure_utility(c)) != IC_OK) {
+    fclose(f);
+    return rc;
+  }
+  // from here on the old contents are gone, whatever happens
+  drop_index(c);
+  c->size = 0;
+  std::vector<unsigned char> bounce(std::min(CKPT_CHUNK, std::max<size_t>(1, (size_t)h.size * c->dim * 2)));
+  rc = copy_device_file(c->slab, (size_t)h.size * c->dim * 2, f, false, bounce, path);
+  if (rc == IC_OK) rc = copy_device_file(c->ids, (size_t)h.size * 8, f, false, bounce, path);
+  if (rc == IC_OK && h.has_utility) rc = copy_device_file(c->utility, (size_t)h.size * 4, f, false, bounce, path);
+  if (rc == IC_OK && !h.has_utility && c->utility && h.size > 0 &&
+      cudaMemset(c->utility, 0, (size_t)h.size * 4) != cudaSuccess)
+    rc = fail(IC_ERR_CUDA, "clearing the utility array failed");
+  fclose(f);
+  if (rc == IC_OK) c->size = h.size;
+  return rc;
+}
+
 int ic_cache_utility_add(ic_cache_t* c, const int64_t* ids_host, const float* gains_host, int64_t n) {
   if (!c) return fail(IC_ERR_INVALID, "NULL handle");
   if (n < 0) return fail(IC_ERR_INVALID, "n %lld < 0", (long long)n);
