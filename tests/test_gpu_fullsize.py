@@ -101,14 +101,19 @@ def test_full_size_workloads_match_the_oracle_on_sampled_queries(loaded):
             assert all(int(i) in set(newest.tolist()) for i in ids[:m, 0].cpu())
 
 
-def test_two_level_search_at_full_size(loaded):
-    """The two-level search on the clustered workload at its full size (after the streaming inserts
-    of the test above, so part of the cache lies outside the index once more rows are appended):
-    index build with K = sqrt(N), then sampled queries against the oracle's two-level definition
-    on the library's own centroids, assignment and probes."""
+def test_two_level_search_at_full_size():
+    """The two-level search on the clustered workload at its full size: index build with
+    K = sqrt(N), then sampled queries against the oracle's two-level definition on the library's
+    own centroids, assignment and probes."""
+    loaded = _Loaded("clustered")
+    try:
+        _two_level_at_full_size(loaded)
+    finally:
+        loaded.close()
+
+
+def _two_level_at_full_size(loaded):
     w = loaded.w
-    if w.name != "clustered":
-        pytest.skip("two-level search is exercised at full size on the clustered workload")
     c = loaded.cache
     c.build_index(0, 3)
     k_clusters, n_indexed = c.index_info()
