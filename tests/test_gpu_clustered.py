@@ -190,6 +190,21 @@ def test_rows_inserted_after_the_build_are_always_searched():
     assert got[0, 0] == ids[20_000] and got[1, 0] == ids[20_017] and got[2, 0] == ids[25_002]
 
 
+@pytest.mark.parametrize("nq,k", [(130, 8), (40, 64)])
+def test_long_tail_of_unindexed_rows(nq, k):
+    # 40,003 rows inserted after the build under a batch of queries: the tiles wholly past the
+    # index (from row 20,224 on) are scored by the tensor-core kernel, rows 20,000 .. 20,223 by
+    # the cluster scan; every row must be searched exactly once
+    w = _blob_workload(20_000, 128, 100, 0.3, seed=309)
+    x = wl.cache_rows(w, DEV)
+    extra = wl.cache_rows(_blob_workload(40_003, 128, 100, 0.3, seed=310), DEV)
+    q = torch.cat([extra[[0, 100, 223, 224, 300, 40_002]], wl.queries(w, nq - 6, DEV)])
+    got, _, _, _ = _clustered_case(x, q, k, 0, 2, 3, extra=extra, what=f"long-tail/nq{nq}")
+    ids = wl.labels(60_003, "cpu")
+    for i, row in enumerate([0, 100, 223, 224, 300, 40_002]):
+        assert got[i, 0] == ids[20_000 + row]
+
+
 def test_fp32_input_and_few_clusters():
     w = wl.WORKLOADS["tiny"]
     x, q = wl.cache_rows(w, DEV), wl.queries(w, 16, DEV)
