@@ -101,7 +101,10 @@ typedef struct ic_cache_plan {
 
 /*
  * Create an empty cache for embeddings of `dim` components with room for `capacity` entries
- * on the current device, input dtype bf16, no normalisation, legacy default stream.
+ * on the current device, input dtype bf16, no normalisation, legacy default stream.  (Paper:
+ * the example cache that IC-Cache's Example Manager owns, Sec. 3 overview and Sec. 4.3; the pool
+ * `examples` that Algorithm 1's GetSimilarExamples searches.  The paper bounds the cache by a
+ * capacity and evicts when it is full; here the capacity is fixed at creation.)
  * dim: multiple of 8, 8 <= dim <= IC_MAX_DIM.  capacity: 1 .. 2^31 - 512.
  * Returns NULL on failure; ic_cache_last_error() then describes why.
  */
@@ -122,7 +125,10 @@ ic_cache_t* ic_cache_create_ex(int32_t dim, int64_t capacity, const ic_cache_opt
 int ic_cache_insert(ic_cache_t* c, const void* emb, const int64_t* ids, int64_t n);
 
 /*
- * For each of nq query embeddings return the k entries with the largest score.
+ * For each of nq query embeddings return the k entries with the largest score.  (Paper:
+ * Algorithm 1, RetrieveExamples stage 1, GetSimilarExamples(request_emb, examples): the
+ * relevance stage of Sec. 4.1, which ranks cached examples by the cosine similarity of dense
+ * request embeddings, best first; the result is the candidate set handed to the stage-2 proxy.)
  * q: [nq, dim] in the handle's input dtype (rounded to bf16 like inserted rows).
  * out_ids [nq, k] int64, out_scores [nq, k] fp32: each row sorted by score descending, equal
  * scores ordered by earlier insertion; when k exceeds the number of entries the tail is
@@ -189,9 +195,12 @@ int ic_cache_query_host(ic_cache_t* c, const void* q_host, int32_t nq, int32_t k
  *   - the first call on a device looks up the array's device address (once per device, with
  *     that device current); make that first call outside any stream capture.
  *   - every handle, stream and thread of the process shares the one array per GPU, and it
- *     keeps the previous call's contents.  Each call writes every word before reading it, so
- *     nothing needs clearing, but two calls whose kernels overlap on the GPU (different
- *     streams or handles) race on the scratch and return garbage: keep them ordered.
+ *     keeps the previous call's contents.  A call writes every data word (staged queries, lists,
+ *     floors, maxima) before it reads it, and the few progress and completion words that CTAs
+ *     of one launch exchange carry a launch number drawn from one counter for the whole
+ *     process, so a word left by an earlier call, of this or any other handle, is never taken
+ *     for a current one: nothing needs clearing.  But two calls whose kernels overlap on the GPU
+ *     (different streams or handles) race on the scratch and return garbage: keep them ordered.
  *   - it calls no cudaMalloc, cudaFree, event creation or other allocating routine, and
  *     ignores ic_cache_set_profiling.
  */
@@ -209,7 +218,7 @@ int ic_cache_insert_host(ic_cache_t* c, const void* emb_host, const int64_t* ids
 
 /*
  * Similarity of cached entries to the OTHER cached entries (the request-similarity study of
- * paper Sec. 2.2: top-1 similarity of each request to the others).  For each of the `count`
+ * paper Sec. 2.2: each request's best match among the other requests).  For each of the `count`
  * entries in slots [first, first+count): the id and score of the best-scoring entry other than
  * itself (an exact copy of it counts as another entry; ties go to the lower slot).
  * out_ids [count] int64, out_scores [count] fp32, device pointers; (-1, -infinity) when the
@@ -313,7 +322,11 @@ int ic_cache_read_index(ic_cache_t* c, void* centroids_host, int64_t* assign_hos
 int ic_cache_query_clustered(ic_cache_t* c, const void* q, int32_t nq, int32_t k, int32_t nprobe,
                              int64_t* out_ids, float* out_scores, int64_t* out_probes);
 
-/* Release the handle and everything the library allocated for it.  NULL is a no-op. */
+/* Release the handle and everything the library allocated for it (synchronises the handle's
+ * stream first; buffers lent through ic_cache_opts_t are left to the caller).  NULL is a no-op.
+ * (Paper Sec. 5, "Fault Tolerance": the serving path keeps working without the retriever, so a
+ * caller may destroy a handle that reported an error and serve without examples, or re-create
+ * it and restore a checkpoint.) */
 void ic_cache_destroy(ic_cache_t* c);
 
 /* Bind the handle to another stream (a cudaStream_t; NULL = legacy default stream).  Work

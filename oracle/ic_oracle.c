@@ -7,8 +7,9 @@
  *   - relevance of a cached example to a request = cosine similarity of their
  *     dense text embeddings (paper Sec. 4.1, "Example Selector", first paragraph;
  *     Sec. 2.2 similarity study: cosine, 1 = identical requests);
- *   - "prioritize examples with high similarity scores" (Sec. 4.1, two-stage
- *     selection paragraph) = return the k best-scoring cached examples;
+ *   - the relevance stage ranks cached examples by that similarity, best first
+ *     (Sec. 4.1, two-stage selection paragraph) = return the k best-scoring
+ *     cached examples;
  *   - Algorithm 1, RetrieveExamples stage 1: GetSimilarExamples(request_emb,
  *     examples).
  * Every score is a brute-force fp32 dot product with the terms added in index
@@ -185,7 +186,7 @@ void ic_oracle_apply_min_score(int64_t* out_ids, float* out_scores, int64_t* out
 
 /*
  * Top-1 similarity of cached entries to the OTHER cached entries (the request-similarity
- * study of paper Sec. 2.2: "top-1 request similarities of each request to others").
+ * study of paper Sec. 2.2: each request's best match among the other requests).
  * For every row i in [first, first+count): the row j != i with the largest fp32 dot product
  * (ties: lowest slot).  out_ids/out_slots/out_scores have `count` entries; with fewer than two
  * rows in the cache the answer is (-1, -1, -inf).  Plain double loop, no blocking.

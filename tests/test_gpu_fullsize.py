@@ -22,7 +22,7 @@ class _Loaded:
     def __init__(self, name):
         self.w = wl.WORKLOADS[name]
         w = self.w
-        rounds = 2 if w.insert_rows else 0
+        rounds = 19 if w.insert_rows else 0
         self.x = wl.cache_rows(w, DEV)
         self.cache = ICCache(w.dim, w.n + rounds * w.insert_rows, input_dtype=wl.torch_dtype(w))
         self.cache.insert(self.x, wl.labels(w.n, DEV))
@@ -88,12 +88,19 @@ def test_full_size_workloads_match_the_oracle_on_sampled_queries(loaded):
         assert plan["n_ctas"] >= 140
         # first, last and two inner queries: with several query tiles this touches the first
         # and the last tile and a tile boundary
-        sample = [0, nq - 1, nq // 2, max(0, min(nq - 1, 128))] if w.n <= 4_000_000 else [0, nq - 1]
+        if w.n <= 4_000_000:
+            sample = [0, nq - 1, nq // 2, max(0, min(nq - 1, 128))]
+        else:
+            # 16 M rows: one query of every 128-query tile (eight oracle queries for the batch of 1024)
+            sample = sorted({min(nq - 1, t * 128 + (37 * t) % 128) for t in range((nq + 127) // 128)} | {0, nq - 1})
         loaded.check(nq, sample)
     if w.insert_rows:
-        # streaming inserts between query batches; planted queries copy rows of the newest batch
-        for rnd in (1, 2):
+        # streaming inserts between query batches; planted queries copy rows of the newest batch.
+        # The oracle re-checks the first rounds and the last of the 20-round timed loop (round 19).
+        for rnd in range(1, 20):
             loaded.append_round(rnd)
+            if rnd not in (1, 2, 19):
+                continue
             ids, sc = loaded.check(w.q_sweep[0], [0, 1, w.planted_queries, w.q_sweep[0] - 1], rnd=rnd)
             m = w.planted_queries
             newest = wl.labels(w.insert_rows, "cpu", first_slot=loaded.n - w.insert_rows)

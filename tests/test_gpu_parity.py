@@ -85,6 +85,28 @@ def test_query_tiling(path, nq, k):
     run_and_check(x, q, k, path=PATHS[path], what=f"qtile/{path}/nq{nq}")
 
 
+@pytest.mark.parametrize("path", ["umma", "auto"])
+@pytest.mark.parametrize("nq", [96, 100, 127, 224, 250, 1000])
+def test_bf16_queries_read_in_place_with_a_partly_filled_last_tile(path, nq):
+    """bf16 queries that need no normalisation are read by the tensor-core kernel straight from the
+    caller's rows when the last 128-query tile is nearly full: the query tensor map then covers
+    fewer rows than its box and the rows past nq must read as zero.  Covers single CTAs (one
+    tile), CTA pairs with a ragged second tile (224, 250) and eight tiles (1000), every query
+    checked against the oracle."""
+    x, q = _gauss(40_003, 256, nq, seed=300 + nq)
+    run_and_check(x, q, 12, path=PATHS[path], what=f"in-place/{path}/nq{nq}")
+
+
+def test_bf16_queries_read_in_place_from_a_16_byte_aligned_pointer():
+    """Same path with a query pointer that is 16-byte but not 128-byte aligned (a view that starts
+    one row into a larger tensor whose rows are 48 bytes long)."""
+    nq, dim = 100, 24
+    x, qq = _gauss(30_001, dim, nq + 1, seed=311)
+    q = qq[1:]
+    assert q.data_ptr() % 16 == 0 and q.data_ptr() % 128 != 0 and q.is_contiguous()
+    run_and_check(x, q, 9, path=IC_PATH_UMMA, what="in-place/offset-pointer")
+
+
 @pytest.mark.parametrize("order", ["random", "best_first", "best_last"])
 @pytest.mark.parametrize("nq,k", [(9, 10), (130, 64), (130, 128), (5, 128)])
 def test_threshold_seeding_pass(order, nq, k):
@@ -410,6 +432,12 @@ def test_random_shapes_tensor_core_path_agrees_with_the_plain_kernel(seed):
         p_ids, p_sc = got["plain"]
         fin = torch.isfinite(p_sc)
         what = f"seed {seed} case {case}: dim {dim} n {n} nq {nq} k {k} {kind}"
+        if n <= 80_000:      # small enough for the oracle: all three paths against it, strictly
+            lab = wl.labels(n).numpy()
+            ref = oracle.search(wl.as_bits(x), wl.as_bits(q), k, ids=lab, want_all_scores=True)
+            for name in ("umma", "auto", "plain"):
+                oracle.accept(got[name][0].numpy(), got[name][1].numpy(), ref["all_scores"], k, ids=lab, tol=1e-4,
+                              what=what + f" [{name} vs oracle]")
         for name in ("umma", "auto"):
             a_ids, a_sc = got[name]
             assert torch.equal(torch.isfinite(a_sc), fin), what
@@ -434,6 +462,7 @@ def test_caller_owned_workspace_serves_queries_without_allocation():
     ids = wl.labels(w.n, DEV)
     need = ic_cache_workspace_bytes(w.dim, w.n, 300, 16)
     ws = torch.empty(need, dtype=torch.uint8, device=DEV)
+    xb, lab = wl.as_bits(x), wl.labels(w.n).numpy()
     with ICCache(w.dim, w.n) as plain, ICCache(w.dim, w.n, workspace=ws) as fixed:
         plain.insert(x, ids)
         fixed.insert(x, ids)
@@ -444,6 +473,10 @@ def test_caller_owned_workspace_serves_queries_without_allocation():
             plain.sync()
             fixed.sync()
             assert torch.equal(a_ids, b_ids) and torch.equal(a_sc, b_sc), f"nq {nq} k {k}"
+            sel = sorted({0, nq // 2, nq - 1})
+            ref = oracle.search(xb, wl.as_bits(q[sel]), k, ids=lab, want_all_scores=True)
+            oracle.accept(b_ids[sel].cpu().numpy(), b_sc[sel].cpu().numpy(), ref["all_scores"], k, ids=lab, tol=1e-4,
+                          what=f"workspace handle nq {nq} k {k}")
         c_ids, c_sc, c_cnt = fixed.query_min_score(wl.queries(w, 7, DEV), 5, 0.12)
         d_ids, d_sc, d_cnt = plain.query_min_score(wl.queries(w, 7, DEV), 5, 0.12)
         assert torch.equal(c_ids, d_ids) and torch.equal(c_cnt, d_cnt)

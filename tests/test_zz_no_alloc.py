@@ -8,6 +8,7 @@ already run every other test."""
 import pytest
 import torch
 
+import oracle
 from paper_2501_12689_b200 import (ICCache, ICCacheError, IC_ERR_NOMEM, IC_ERR_INVALID, IC_PATH_AUTO,
                                    IC_PATH_GENERIC, workloads as wl)
 from parity_util import TOL_STRICT
@@ -28,12 +29,25 @@ def _case(n, dim, nq, k, seed, path=IC_PATH_AUTO):
         # caller-owned outputs, allocated before the calls under test
         outs = [(torch.empty(nq, k, dtype=torch.int64, device=DEV),
                  torch.empty(nq, k, dtype=torch.float32, device=DEV)) for _ in range(2)]
+        c.query_static(q1, k, *outs[0])      # first use on this GPU looks the array's address up
+        c.sync()
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         c.query_static(q1, k, *outs[0])      # two calls in a row share the static scratch
         c.query_static(q2, k, *outs[1])
         c.sync()
+        # nothing was allocated on the device by the two calls (torch allocated nothing either:
+        # every tensor above exists already)
+        assert torch.cuda.mem_get_info()[0] == free_before
         for (wi, ws), (gi, gs) in zip(want, outs):
             assert torch.equal(wi, gi)
             assert torch.allclose(ws, gs, atol=TOL_STRICT, rtol=0)
+        # and against the CPU oracle, strictly
+        lab = wl.labels(n).numpy()
+        for q, (gi, gs) in zip((q1, q2), outs):
+            ref = oracle.search(wl.as_bits(x), wl.as_bits(q), k, ids=lab, want_all_scores=True)
+            oracle.accept(gi.cpu().numpy(), gs.cpu().numpy(), ref["all_scores"], k, ids=lab, tol=TOL_STRICT,
+                          what=f"static scratch n {n} dim {dim} nq {nq} k {k}")
 
 
 def test_static_query_matches_query_scan_path():
