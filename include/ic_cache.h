@@ -81,7 +81,8 @@ typedef struct ic_cache_opts {
 /* Host-side launch plan for one query call; pure function of its arguments. */
 typedef struct ic_cache_plan {
   int32_t path;          /* ic_path actually used                                          */
-  int32_t query_tile;    /* queries handled together by one CTA                            */
+  int32_t query_tile;    /* queries handled together by one CTA (tensor cores: 128, or 64
+                            with a resident query tile)                                    */
   int32_t n_query_tiles; /* per launch                                                     */
   int32_t n_partitions;  /* row partitions = partial top-k lists per query                 */
   int32_t n_ctas;        /* CTAs of the scoring kernel                                     */
@@ -92,11 +93,14 @@ typedef struct ic_cache_plan {
   int32_t seed_tiles;    /* tensor-core path: 256-row tiles scored into lists ahead of the
                             main pass, whose merged k-th key is the main pass's floor; the
                             main pass skips them (0 = none)                                */
-  int32_t seed0_tiles;   /* tensor-core path: tiles of a maxima-only launch whose k-th
-                            largest group maximum per query is the first floor; these
-                            tiles are scored again afterwards (0 = none)                   */
+  int32_t seed0_tiles;   /* tensor-core path: tiles (the first few of every partition, about
+                            one per SM in all) whose group maxima the CTAs of a launch
+                            exchange to agree on a first floor per query (0 = no seeding
+                            inside the launch)                                             */
   int32_t cta_group;     /* tensor-core path: 2 = CTA pairs issue one 256-query MMA and
                             split each row tile between them, 1 = single CTAs (else 0)     */
+  int32_t query_resident;/* tensor-core path: 1 = at most 64 queries, M = 64, the whole query
+                            tile stays in shared memory and ring stages hold cache rows only */
 } ic_cache_plan_t;
 
 /*
@@ -181,7 +185,7 @@ int ic_cache_query_host(ic_cache_t* c, const void* q_host, int32_t nq, int32_t k
  * late cudaMalloc fails), or a latency-critical loop whose rules forbid calls that may
  * synchronise the device, which cudaMalloc and cudaFree do.  ic_cache_query grows the
  * library's scratch buffers on the first call of a larger shape; this variant never does.
- * Its scratch (query staging, partial top-k lists, seed thresholds, group maxima) is carved out of one
+ * Its scratch (query staging, partial top-k lists, seed thresholds, group maxima, progress words) is carved out of one
  * fixed array of IC_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that
  * loads the library holds that much memory until the process exits, whether or not this
  * call is ever used.
@@ -364,8 +368,8 @@ int64_t ic_cache_launch_count(const ic_cache_t* c);
  * Measurement aid.  While enabled, the launches of this handle are bracketed by pairs of CUDA
  * events on the handle's stream, in three groups: "scoring" = the scan launch(es), or the main
  * pass of the tensor-core path (the launch that reads all rows outside the list-level sample);
- * "seed" = each threshold-seeding launch together with the selection or merge that turns its
- * output into per-query floors; "merge" = the final merge.  At most 16384 brackets of each group between two reads; later ones go
+ * "seed" = the launch that scores the list-level sample of a large cache together with the merge
+ * that turns its lists into per-query floors; "merge" = the final merge.  At most 16384 brackets of each group between two reads; later ones go
  * unrecorded.  ic_cache_query_static records nothing.
  */
 int ic_cache_set_profiling(ic_cache_t* c, int32_t enable);

@@ -43,7 +43,7 @@ class ic_cache_opts_t(ctypes.Structure):
 class ic_cache_plan_t(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "path", "query_tile", "n_query_tiles", "n_partitions", "n_ctas", "n_stages", "smem_bytes",
-        "n_launches", "queue_cap", "seed_tiles", "seed0_tiles", "cta_group")]
+        "n_launches", "queue_cap", "seed_tiles", "seed0_tiles", "cta_group", "query_resident")]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}

@@ -10,6 +10,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <atomic>
 #include <mutex>
 #include <new>
 #include <vector>
@@ -33,7 +34,8 @@ constexpr int WINDOW_MAX_NQ = 1024;   // queries scored per pass over the slab
 constexpr int QUERY_TILE = 128;       // tcgen05 path: queries per CTA (MMA M)
 constexpr int ROW_TILE = 256;         // tcgen05 path: cache rows per accumulator (MMA N)
 constexpr int K_CHUNK = 64;           // tcgen05 path: bf16 elements per 128-byte swizzled row
-constexpr int UMMA_STAGE_BYTES = (QUERY_TILE + ROW_TILE) * K_CHUNK * 2;  // 48 KiB
+constexpr int RESIDENT_MAX_NQ = 64;   // tcgen05 path: batches up to this size keep their query tile in shared memory
+constexpr int RESIDENT_MIN_STAGES = 4;
 constexpr int SCAN_MAX_Q = 4;        // queries per scan launch
 constexpr int SCAN_AUTO_MAX_Q = 2;   // largest batch the automatic choice gives to the scan path
 constexpr int SCAN_MAX_DIM = 1024;
@@ -45,7 +47,18 @@ constexpr int SEED_MIN_TILES_PER_CTA = 8;  // tcgen05 path: seed thresholds when
 constexpr int SEED_FRACTION = 16;          // share of the row tiles scored by the seeding pass
 constexpr int SEED_TWO_LEVEL_TILES_PER_CTA = 4;
 constexpr int64_t DENSE_TAIL_MIN_ROWS = 1024;   // two-level search: rows past the index from which they go to the tensor-core kernel
-constexpr size_t PACE_BYTES = 16384;       // progress words of the tensor-core path: one per CTA, 2048 at most
+// Words that the CTAs of one tensor-core launch exchange: 8 KiB of progress words (L2 pacing, one per
+// CTA or pair) followed by 8 KiB of seeding flags (one per CTA).  Every word carries the launch's
+// number, drawn from one counter for the whole process, so words of earlier launches (of any handle
+// that shares the block) are never taken for current ones.
+constexpr size_t PACE_BYTES = 16384;
+constexpr size_t SEED_FLAGS_OFFSET = 8192;
+std::atomic<unsigned> g_launch_epoch{0};
+unsigned next_epoch() {
+  unsigned e = ++g_launch_epoch;
+  if (e == 0) e = ++g_launch_epoch;   // 0 is what a cleared word holds
+  return e;
+}
 
 struct DeviceGuard {
   int prev = -1;
@@ -86,7 +99,6 @@ struct ic_cache {
   int64_t* ids = nullptr;
   bool own_ids = false;
   Buffer q_bf16, q_f32, partials, thr, maxima, pace, stage_in, stage_ids, stage_scores, evict;
-  unsigned pace_epoch = 0;
   int l2_bytes = 0;
   int* h_status = nullptr;  // pinned, mapped; kernels write a code when a bounded wait expires
   int* d_status = nullptr;
@@ -101,6 +113,8 @@ struct ic_cache {
   float* utility = nullptr;   // [capacity] per-entry utility, allocated on first use, zero for new entries
   Buffer util_ids, util_gains;
   Buffer idx_assign, idx_best, idx_order, idx_offsets, idx_sort, idx_init, idx_probes, idx_probe_scores;
+  Buffer idx_rows;            // cluster-contiguous copy of the indexed rows (optional: absent if memory is short)
+  bool have_idx_rows = false;
   EncodeTiledFn encode = nullptr;
   CUtensorMap tmap_slab;       // box of 256 rows
   CUtensorMap tmap_slab_half;  // box of 128 rows, for CTA pairs
@@ -214,47 +228,65 @@ int plan_impl(int32_t dim, int64_t n, int32_t nq, int32_t k, int32_t path, int32
     const int units = out->n_query_tiles / out->cta_group;                    // CTAs or pairs per partition
     out->n_partitions = std::max(1, std::min((sm_count / out->cta_group) / units, merge_lists_max - 1));
     out->n_ctas = out->n_partitions * out->n_query_tiles;
-    // Threshold seeding, with enough row tiles per CTA.  Level 0 (seed0_tiles): a maxima-only
-    // launch over about one tile per SM gives, per query, the k-th largest of the group maxima,
-    // a floor for its top-k; those tiles are scored again by the next launch.  Level 1
-    // (seed_tiles, large caches only): 1/16 of the tiles are scored with that floor into real
-    // lists, whose merge gives the sample's exact k-th key as the floor of the main pass, which
-    // then skips the sampled tiles.
+    // Threshold seeding, with enough row tiles per CTA.  Level 0 (seed0_tiles, about one tile per
+    // SM) happens inside the scoring launch: every CTA publishes the group maxima of its first
+    // tiles and takes, per query, (about) the k-th largest of all of them as a floor.  Level 1
+    // (seed_tiles, large caches only): 1/16 of the tiles are scored first, by a launch of their
+    // own, into real lists, whose merge gives the sample's exact k-th key as the floor of the
+    // main pass, which then skips the sampled tiles.
     const int64_t n_tiles = (n + ROW_TILE - 1) / ROW_TILE;
-    const char* seed_env = getenv("IC_CACHE_SEED");   // tuning knob: "0" scores everything in one pass
-    // A handful of queries with short lists does better without: few lanes of a warp are real, so
-    // passing columns are rare anyway, and the cold-start floor of the first tile (k <= 16) is
-    // cheap (measured at N = 1 M, k = 10: 247 against 271 us per step for 3 queries, 267 against
-    // 272 for 8, 295 against 273 for 16).
-    const bool seeding = !(seed_env && seed_env[0] == '0' && seed_env[1] == 0) && !(window <= 8 && k <= 16);
-    const int t0 = (sm_count + out->n_partitions - 1) / out->n_partitions;   // level-0 tiles per partition
-    const int64_t level0 = (int64_t)t0 * out->n_partitions;
-    if (seeding && n_tiles >= (int64_t)SEED_MIN_TILES_PER_CTA * out->n_partitions && n / ROW_TILE >= level0 &&
-        level0 * 4 >= k && level0 * 4 <= 1280) {
-      out->seed0_tiles = (int32_t)level0;
+    const char* seed_env = getenv("IC_CACHE_SEED");   // tuning knob: "0" scores everything in one pass, unseeded
+    const bool seeding = !(seed_env && seed_env[0] == '0' && seed_env[1] == 0);
+    const int P = out->n_partitions;
+    if (seeding && n_tiles >= (int64_t)SEED_MIN_TILES_PER_CTA * P) {
       int seed_fraction = SEED_FRACTION;
       if (const char* fe = getenv("IC_CACHE_SEED_FRACTION")) {   // tuning knob: 1/fraction of the tiles are sampled
         const int f = atoi(fe);
         if (f >= 2) seed_fraction = f;
       }
-      const int64_t t = n_tiles / seed_fraction / out->n_partitions * out->n_partitions;
-      if (t >= (int64_t)SEED_TWO_LEVEL_TILES_PER_CTA * out->n_partitions && t > level0) out->seed_tiles = (int32_t)t;
+      const int64_t t = n_tiles / seed_fraction / P * P;
+      if (t >= (int64_t)SEED_TWO_LEVEL_TILES_PER_CTA * P && t > P) out->seed_tiles = (int32_t)t;
+      // tiles per CTA whose maxima are exchanged inside the (first) launch: about one tile per SM
+      // in all, so that the sample does not shrink when there are few partitions
+      const int64_t first_launch_tiles = out->seed_tiles > 0 ? out->seed_tiles : n / ROW_TILE;   // full tiles only
+      const int64_t t0 = std::min<int64_t>({(sm_count + P - 1) / P, 16, first_launch_tiles / P});
+      if (t0 >= 1 && t0 * P * 4 >= k) out->seed0_tiles = (int32_t)(t0 * P);
+      else out->seed_tiles = 0;   // no first floor: the sample launch would start cold
     }
-    // 1 KiB alignment slack + 256 B of barriers, the per-query lists, then as many candidate
-    // queue entries per query (up to 8) as still leave room for two ring stages
-    const int base = 1024 + 256 + QUERY_TILE * k * 8;
-    const int stage_bytes = (QUERY_TILE + ROW_TILE / out->cta_group) * K_CHUNK * 2;   // 48 or 32 KiB
-    out->queue_cap = std::min(8, (smem_optin - base - 2 * stage_bytes) / (QUERY_TILE * 8));
-    if (out->queue_cap < 1) return fail(IC_ERR_UNSUPPORTED, "tensor-core path: shared memory too small");
-    const int fixed = base + QUERY_TILE * out->queue_cap * 8;
-    out->n_stages = std::min(8, (smem_optin - fixed) / stage_bytes);
+    // Shared memory: as many candidate queue entries per query (up to 8) as still leave room for the
+    // smallest ring, then as many ring stages as fit.  Batches of at most 64 queries keep their whole
+    // query tile resident (M = 64) when that still leaves a ring of four 16 KiB stages.
+    int max_stages = 12;
     if (const char* env = getenv("IC_CACHE_MAX_STAGES")) {   // tuning knob: cap on the ring depth
       const int cap = atoi(env);
-      if (cap >= 2) out->n_stages = std::min(out->n_stages, cap);
+      if (cap >= 2) max_stages = std::min(max_stages, cap);
     }
-    if (out->n_stages < 2) return fail(IC_ERR_UNSUPPORTED, "tensor-core path: shared memory too small");
-    out->smem_bytes = fixed + out->n_stages * stage_bytes;
-    out->n_launches = n_windows * (1 + (out->seed_tiles > 0 ? 1 : 0) + (out->seed0_tiles > 0 ? 1 : 0));
+    auto fit = [&](bool resident, int min_stages, int* qcap, int* stages) {
+      for (int qc = 8; qc >= 1; --qc) {
+        if (icc::umma_smem_bytes(out->cta_group, resident, dim, k, qc, min_stages) > (size_t)smem_optin) continue;
+        int st = min_stages;
+        while (st < max_stages && icc::umma_smem_bytes(out->cta_group, resident, dim, k, qc, st + 1) <= (size_t)smem_optin) ++st;
+        *qcap = qc;
+        *stages = st;
+        return true;
+      }
+      return false;
+    };
+    const char* qres_env = getenv("IC_CACHE_QRES");   // tuning knob: "0" streams the query tile for every batch size
+    const bool want_resident = window <= RESIDENT_MAX_NQ && !(qres_env && qres_env[0] == '0' && qres_env[1] == 0);
+    int qcap = 0, stages = 0;
+    if (want_resident && fit(true, std::min(RESIDENT_MIN_STAGES, max_stages), &qcap, &stages)) {
+      out->query_resident = 1;
+      out->query_tile = RESIDENT_MAX_NQ;
+    } else if (!fit(false, 2, &qcap, &stages)) {
+      return fail(IC_ERR_UNSUPPORTED, "tensor-core path: shared memory too small");
+    }
+    // twice the queue (fewer drains) when it costs no ring stage
+    if (qcap == 8 && icc::umma_smem_bytes(out->cta_group, out->query_resident != 0, dim, k, 16, stages) <= (size_t)smem_optin) qcap = 16;
+    out->queue_cap = qcap;
+    out->n_stages = stages;
+    out->smem_bytes = (int32_t)icc::umma_smem_bytes(out->cta_group, out->query_resident != 0, dim, k, qcap, stages);
+    out->n_launches = n_windows * (1 + (out->seed_tiles > 0 ? 1 : 0));
   }
   return IC_OK;
 }
@@ -309,10 +341,17 @@ int ensure_utility(ic_cache* c) {
   return IC_OK;
 }
 
-// Tensor-core scoring of one window: an optional maxima-only launch over seed0_tiles tiles whose
-// group maxima give a first floor per query (select kernel), an optional launch over the first
-// seed_tiles tiles into real lists whose merge gives the sample's exact k-th key, then the main
-// pass over the tiles not yet in a list.  Lists are blocks of nq*k keys inside `partials`:
+// Bytes of group maxima that seeding inside a tensor-core launch exchanges: four floats per
+// (query tile, partition, tensor-memory lane).
+size_t seed_maxima_bytes(const ic_cache_plan_t& pl) {
+  return (size_t)pl.n_query_tiles * pl.seed0_tiles * QUERY_TILE * 16;
+}
+
+// Tensor-core scoring of one window.  Large caches: a launch over the first seed_tiles tiles into
+// real lists, whose merge gives the sample's exact k-th key per query as the floor of the main
+// pass; then the main pass over the tiles not yet in a list.  A launch that is given no floors
+// seeds itself from the group maxima of its CTAs' first tiles (seed0_tiles > 0).  Lists are blocks
+// of nq*k keys inside `partials`:
 //   blocks 0 .. P-1      main pass            block P          merged sample list
 //   blocks P+1 .. 2P     lists of the sampling launch
 // On return *n_final_lists tells the final merge how many leading blocks to read.
@@ -323,14 +362,14 @@ int run_umma_passes(ic_cache* c, const ic_cache_plan_t& pl, const void* q_bf16, 
   const int P = pl.n_partitions;
   const size_t list_block = (size_t)nq * k;
   icc::UmmaParams up;
-  int rc = encode_2d(c, &up.tmap_q, q_bf16, (uint64_t)nq_pad, QUERY_TILE);
+  int rc = encode_2d(c, &up.tmap_q, q_bf16, (uint64_t)nq_pad, pl.query_resident ? RESIDENT_MAX_NQ : QUERY_TILE);
   if (rc != IC_OK) return rc;
   up.tmap_slab = c->tmap_slab;
   up.tmap_slab_half = c->tmap_slab_half;
   up.cta_group = pl.cta_group;
+  up.q_resident = pl.query_resident;
   up.n = c->size;
   up.dim = c->dim;
-  up.q0 = 0;
   up.nq = nq;
   up.k = k;
   up.n_query_tiles = pl.n_query_tiles;
@@ -339,6 +378,7 @@ int run_umma_passes(ic_cache* c, const ic_cache_plan_t& pl, const void* q_bf16, 
   up.queue_cap = pl.queue_cap;
   up.smem_bytes = pl.smem_bytes;
   up.dev_status = c->d_status;
+  up.seed_t0 = pl.seed0_tiles / P;
   // CTAs of one partition may run an eighth of the partition's share of L2 apart (measured: with
   // 18 partitions of 393 KB tiles, 3 tiles keep DRAM reads at the slab size, 8 tiles do not)
   up.pace = pace;
@@ -352,38 +392,24 @@ int run_umma_passes(ic_cache* c, const ic_cache_plan_t& pl, const void* q_bf16, 
   const int64_t n_tiles = (c->size + ROW_TILE - 1) / ROW_TILE;
   uint64_t* pass_lists = partials + (size_t)(P + 1) * list_block;
   uint64_t* merged = partials + (size_t)P * list_block;
-  bool have_thr = false;
-  int64_t begin = 0;
-  *n_final_lists = P;
-  cudaError_t e;
   // only_from_tile >= 0: a single launch over the tiles from there on, no seeding (the two-level
   // search uses it for the rows inserted after its index was built)
   const bool whole = only_from_tile < 0;
-  if (!whole) begin = only_from_tile;
-  if (whole && pl.seed0_tiles > 0 && maxima) {
-    up.tile_begin = 0;
-    up.tile_end = pl.seed0_tiles;
-    up.thr_floor = nullptr;
-    up.partials = nullptr;
-    up.maxima_out = maxima;
-    up.pace_epoch = ++c->pace_epoch;
-    if (profile) profile_mark(c, c->ev_seed, c->n_ev_seed);
-    e = icc::launch_umma(up, c->stream);
-    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core maxima launch failed: %s", cudaGetErrorString(e));
-    c->launches += 1;
-    e = icc::launch_select_floor(maxima, pl.seed0_tiles, nq, k, thr, c->stream);
-    if (e != cudaSuccess) return fail(IC_ERR_CUDA, "floor selection launch failed: %s", cudaGetErrorString(e));
-    c->launches += 1;
-    if (profile) profile_mark(c, c->ev_seed, c->n_ev_seed);
-    have_thr = true;   // the tiles themselves are scored again below
-  }
-  up.maxima_out = nullptr;
+  // seeding inside a launch: its flags sit behind the progress words
+  const bool self_seed = whole && pl.seed0_tiles > 0 && maxima != nullptr && pace != nullptr;
+  unsigned* flags = reinterpret_cast<unsigned*>(reinterpret_cast<unsigned char*>(pace) + SEED_FLAGS_OFFSET);
+  bool have_thr = false;
+  int64_t begin = whole ? 0 : only_from_tile;
+  *n_final_lists = P;
+  cudaError_t e;
   if (whole && pl.seed_tiles > 0) {
     up.tile_begin = 0;
     up.tile_end = pl.seed_tiles;
-    up.thr_floor = have_thr ? thr : nullptr;
+    up.thr_floor = nullptr;
     up.partials = pass_lists;
-    up.pace_epoch = ++c->pace_epoch;
+    up.seed_maxima = self_seed ? maxima : nullptr;
+    up.seed_flags = self_seed ? flags : nullptr;
+    up.epoch = next_epoch();
     if (profile) profile_mark(c, c->ev_seed, c->n_ev_seed);
     e = icc::launch_umma(up, c->stream);
     if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core sampling launch failed: %s", cudaGetErrorString(e));
@@ -400,7 +426,9 @@ int run_umma_passes(ic_cache* c, const ic_cache_plan_t& pl, const void* q_bf16, 
   up.tile_end = n_tiles;
   up.thr_floor = have_thr ? thr : nullptr;
   up.partials = partials;
-  up.pace_epoch = ++c->pace_epoch;
+  up.seed_maxima = (self_seed && !have_thr) ? maxima : nullptr;
+  up.seed_flags = (self_seed && !have_thr) ? flags : nullptr;
+  up.epoch = next_epoch();
   if (profile) profile_mark(c, c->ev_score, c->n_ev_score);
   e = icc::launch_umma(up, c->stream);
   if (e != cudaSuccess) return fail(IC_ERR_CUDA, "tensor-core scoring launch failed: %s", cudaGetErrorString(e));
@@ -422,15 +450,18 @@ int do_query_window(ic_cache* c, const void* q, int nq, int k, int64_t* out_ids,
   const size_t list_block = (size_t)nq * k;   // keys of one partition
   if ((rc = ensure(c, c->partials, (size_t)(2 * pl.n_partitions + 2) * list_block * 8, "partial top-k lists")) != IC_OK) return rc;
   if ((rc = ensure(c, c->thr, (size_t)nq * 8, "seed thresholds")) != IC_OK) return rc;
-  if ((rc = ensure(c, c->maxima, (size_t)pl.seed0_tiles * nq * 16, "group maxima")) != IC_OK) return rc;
+  if ((rc = ensure(c, c->maxima, seed_maxima_bytes(pl), "group maxima")) != IC_OK) return rc;
 
   // bf16 queries that need no normalisation go to the tensor-core path as they are: the query
   // tensor map points at the caller's rows and rows past nq read as zero, so the conversion
-  // launch (and its place in the chain of dependent kernels) is saved.  Only with the last query
-  // tile nearly full: out-of-range rows load slowly (measured main pass, 500-step runs: 64 queries
+  // launch (and its place in the chain of dependent kernels) is saved.  With a streamed query
+  // tile only when its last 128 rows are nearly all there: out-of-range rows load slowly, and
+  // they would be loaded with every ring stage (measured main pass, 500-step runs: 64 queries
   // 240 -> 262 us, 16 queries 221 -> 261 us; 100 and 128 queries unchanged, step 2-4 us shorter).
+  // A resident query tile is loaded once per CTA, so there it always pays.
   const bool direct = pl.path == IC_PATH_UMMA && c->input_dtype == IC_BF16 && !c->normalize &&
-                      (reinterpret_cast<uintptr_t>(q) & 15) == 0 && nq_pad - nq <= QUERY_TILE / 4;
+                      (reinterpret_cast<uintptr_t>(q) & 15) == 0 &&
+                      (pl.query_resident || nq_pad - nq <= QUERY_TILE / 4);
   cudaError_t e = cudaSuccess;
   if (!direct) {
     e = icc::launch_convert_rows(q, c->input_dtype == IC_F32, nq, c->dim, c->normalize, c->q_bf16.p,
@@ -523,13 +554,13 @@ FixedLayout fixed_layout(int dim, int nq, int k, const ic_cache_plan_t& pl) {
   const size_t list_block = (size_t)nq * k;
   auto round_up = [](size_t v) { return (v + 1023) & ~(size_t)1023; };
   FixedLayout f;
-  f.off_qbf16 = 0;
+  f.off_pace = 0;   // at a fixed place, whatever the shape
+  f.off_qbf16 = PACE_BYTES;
   f.off_qf32 = f.off_qbf16 + round_up((size_t)nq_pad * dim * 2);
   f.off_part = f.off_qf32 + round_up((size_t)nq * dim * 4);
   f.off_thr = f.off_part + round_up((size_t)(2 * pl.n_partitions + 2) * list_block * 8);
   f.off_max = f.off_thr + round_up((size_t)nq * 8);
-  f.off_pace = f.off_max + round_up((size_t)pl.seed0_tiles * nq * 16);
-  f.need = f.off_pace + PACE_BYTES;
+  f.need = f.off_max + round_up(seed_maxima_bytes(pl));
   return f;
 }
 
@@ -612,7 +643,7 @@ int query_bf16_rows(ic_cache* c, const char* q_rows, int64_t count, int64_t read
     const size_t list_block = (size_t)nq * k;
     if ((rc = ensure(c, c->partials, (size_t)(2 * pl.n_partitions + 2) * list_block * 8, "partial top-k lists")) != IC_OK) return rc;
     if ((rc = ensure(c, c->thr, (size_t)nq * 8, "seed thresholds")) != IC_OK) return rc;
-    if ((rc = ensure(c, c->maxima, (size_t)pl.seed0_tiles * nq * 16, "group maxima")) != IC_OK) return rc;
+    if ((rc = ensure(c, c->maxima, seed_maxima_bytes(pl), "group maxima")) != IC_OK) return rc;
     uint64_t* partials = static_cast<uint64_t*>(c->partials.p);
     int n_final_lists = 0;
     // the map may cover following rows up to a full 128-row tile, never past `readable`; lanes
@@ -639,6 +670,7 @@ void drop_index(ic_cache* c) {
   }
   c->n_clusters = 0;
   c->n_indexed = 0;
+  c->have_idx_rows = false;
 }
 
 int check_query_args(ic_cache* c, const void* q, int32_t nq, int32_t k, const void* out_ids, const void* out_scores) {
@@ -753,6 +785,11 @@ ic_cache_t* ic_cache_create_ex(int32_t dim, int64_t capacity, const ic_cache_opt
     if (!is_device_ptr(o.workspace, dev) || (reinterpret_cast<uintptr_t>(o.workspace) & 255)) {
       fail(IC_ERR_INVALID, "opts.workspace must be a 256-byte aligned device pointer on device %d", dev);
       ok = false;
+    } else if (c->workspace_bytes >= PACE_BYTES && cudaMemset(o.workspace, 0, PACE_BYTES) != cudaSuccess) {
+      // the words the CTAs of a launch exchange start out cleared
+      cudaGetLastError();
+      fail(IC_ERR_CUDA, "clearing the head of opts.workspace failed");
+      ok = false;
     }
   }
   if (ok) {
@@ -849,6 +886,7 @@ void ic_cache_destroy(ic_cache_t* c) {
   release(c->idx_init);
   release(c->idx_probes);
   release(c->idx_probe_scores);
+  release(c->idx_rows);
   if (c->own_slab && c->slab) cudaFree(c->slab);
   if (c->own_ids && c->ids) cudaFree(c->ids);
   release(c->q_bf16);
@@ -1314,6 +1352,11 @@ int ic_cache_build_index(ic_cache_t* c, int32_t n_clusters, int32_t n_iters, con
   }
   child->size = K;
   child->launches += 1;
+  // one status word for parent and child: a bounded wait that expires in a kernel launched through
+  // the child (assignment passes, a query's centroid step) is reported by the parent's calls
+  if (child->h_status) cudaFreeHost(child->h_status);
+  child->h_status = nullptr;
+  child->d_status = c->d_status;
   int64_t* assign = static_cast<int64_t*>(c->idx_assign.p);
   for (int it = 0; it <= n_iters && rc == IC_OK; ++it) {
     // assignment: every cached row is a query against the centroids, best centroid per row
@@ -1327,6 +1370,20 @@ int ic_cache_build_index(ic_cache_t* c, int32_t n_clusters, int32_t n_iters, con
                                       static_cast<const int*>(c->idx_order.p), (int)K, child->slab, c->stream);
     if (e != cudaSuccess) rc = fail(IC_ERR_CUDA, "clustering launch failed: %s", cudaGetErrorString(e));
     child->launches += it < n_iters ? 5 : 4;
+  }
+  // Cluster-contiguous copy of the rows, so that a probed cluster is one contiguous run to stream.
+  // It costs as much memory again as the indexed rows; when that is not to be had the search
+  // fetches rows through the member lists instead (slower, same results).
+  c->have_idx_rows = false;
+  if (rc == IC_OK) {
+    if (ensure(c, c->idx_rows, (size_t)n * c->dim * 2, "cluster-contiguous rows") == IC_OK) {
+      e = icc::launch_gather_by_order(c->slab, static_cast<const int*>(c->idx_order.p), n, c->dim, c->idx_rows.p, c->stream);
+      if (e != cudaSuccess) rc = fail(IC_ERR_CUDA, "row gather launch failed: %s", cudaGetErrorString(e));
+      else c->have_idx_rows = true;
+      child->launches += 1;
+    } else {
+      g_err[0] = 0;
+    }
   }
   if (rc == IC_OK && cudaStreamSynchronize(c->stream) != cudaSuccess) rc = fail(IC_ERR_CUDA, "clustering failed on the device");
   if (rc == IC_OK) rc = check_timeout(c);
@@ -1375,7 +1432,6 @@ int ic_cache_query_clustered(ic_cache_t* c, const void* q, int32_t nq, int32_t k
     return fail(IC_ERR_INVALID, "q, out_ids, out_scores and out_probes must be device pointers on device %d", c->device);
   if ((rc = check_timeout(c)) != IC_OK) return rc;
   const int np = nprobe;   // probes past the number of clusters come back as -1 and give empty lists
-  const int64_t tail = c->size - c->n_indexed;
   const size_t q_row = (size_t)c->dim * in_elem_bytes(c);
   const int merge_lists_max = (c->smem_optin - 4096) / (k * 8 + 4);
   for (int q0 = 0; q0 < nq; q0 += WINDOW_MAX_NQ) {
@@ -1423,7 +1479,7 @@ int ic_cache_query_clustered(ic_cache_t* c, const void* q, int32_t nq, int32_t k
     cudaError_t e = icc::launch_convert_rows(qw, c->input_dtype == IC_F32, w, c->dim, c->normalize, c->q_bf16.p,
                                              static_cast<float*>(c->q_f32.p), nq_pad, nullptr, nullptr, c->stream);
     if (e == cudaSuccess)
-      e = icc::launch_cluster_scan(c->slab, scan_end, c->dim, static_cast<const float*>(c->q_f32.p), w, k, probes, nprobe,
+      e = icc::launch_cluster_scan(c->slab, c->have_idx_rows ? c->idx_rows.p : nullptr, scan_end, c->dim, static_cast<const float*>(c->q_f32.p), w, k, probes, nprobe,
                                    n_split, n_tail, static_cast<const int*>(c->idx_offsets.p),
                                    static_cast<const int*>(c->idx_order.p), c->n_indexed,
                                    static_cast<uint64_t*>(c->partials.p), c->stream);

@@ -34,6 +34,27 @@ cudaError_t launch_gather_rows(const void* slab, const int64_t* slots, int n_row
   return cudaGetLastError();
 }
 
+// Cluster-contiguous copy of the indexed rows: row p of out_rows is cache row order[p], so the
+// members of a cluster are one contiguous run that the two-level search streams.  One warp per row.
+__global__ void __launch_bounds__(256)
+gather_by_order_kernel(const __nv_bfloat16* __restrict__ slab, const int* __restrict__ order, int64_t n_rows, int dim,
+                       __nv_bfloat16* __restrict__ out_rows) {
+  const int lane = threadIdx.x & 31;
+  const int64_t p = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (p >= n_rows) return;
+  const uint4* from = reinterpret_cast<const uint4*>(slab + (int64_t)order[p] * dim);
+  uint4* to = reinterpret_cast<uint4*>(out_rows + p * dim);
+  for (int v = lane; v < (dim >> 3); v += 32) to[v] = ld_stream_16B(from + v);
+}
+
+cudaError_t launch_gather_by_order(const void* slab, const int* order, int64_t n_rows, int dim, void* out_rows,
+                                   cudaStream_t st) {
+  if (n_rows <= 0) return cudaSuccess;
+  gather_by_order_kernel<<<(unsigned)((n_rows + 7) / 8), 256, 0, st>>>(static_cast<const __nv_bfloat16*>(slab), order, n_rows,
+                                                                        dim, static_cast<__nv_bfloat16*>(out_rows));
+  return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------ stable counting sort
 // Rows are cut into blocks of SORT_ROWS_PER_BLOCK consecutive slots.
 //   1. hist:    blk_hist[b][c] = rows of block b assigned to cluster c
@@ -260,10 +281,10 @@ constexpr int CS_WARPS = 8;
 constexpr int CS_ROWS = 4;    // rows in flight per warp
 
 __global__ void __launch_bounds__(CS_WARPS * 32)
-cluster_scan_topk_kernel(const __nv_bfloat16* __restrict__ slab, int64_t n, int dim, const float* __restrict__ q_f32,
-                         int nq, int k, const int64_t* __restrict__ probes, int n_probe, int n_split, int n_tail,
-                         const int* __restrict__ offsets, const int* __restrict__ order, int64_t n_indexed,
-                         uint64_t* __restrict__ partials) {
+cluster_scan_topk_kernel(const __nv_bfloat16* __restrict__ slab, const __nv_bfloat16* __restrict__ sorted_rows, int64_t n,
+                         int dim, const float* __restrict__ q_f32, int nq, int k, const int64_t* __restrict__ probes,
+                         int n_probe, int n_split, int n_tail, const int* __restrict__ offsets,
+                         const int* __restrict__ order, int64_t n_indexed, uint64_t* __restrict__ partials) {
   extern __shared__ __align__(16) unsigned char cs_smem[];
   float* qs = reinterpret_cast<float*>(cs_smem);                         // [dim]
   uint64_t* lists = reinterpret_cast<uint64_t*>(qs + dim);               // [CS_WARPS][k]
@@ -298,15 +319,18 @@ cluster_scan_topk_kernel(const __nv_bfloat16* __restrict__ slab, int64_t n, int 
   uint64_t thr = KEY_EMPTY;
   const int n_chunks = dim >> 3;
   for (int64_t m = m0 + CS_ROWS * warp; m < m1; m += CS_ROWS * CS_WARPS) {
-    // CS_ROWS rows per warp and step: all their loads are issued before the first product
-    int64_t slot[CS_ROWS];
+    // CS_ROWS rows per warp and step: all their loads are issued before the first product.  With a
+    // cluster-contiguous copy of the rows the members of a cluster are read in place, one after
+    // the other, and a row's slot is looked up in the member list only if its score can enter
+    // the list; without one every row is fetched through the member list.
+    int64_t pos[CS_ROWS];
     const uint4* row[CS_ROWS];
     float acc[CS_ROWS];
 #pragma unroll
     for (int r = 0; r < CS_ROWS; ++r) {
-      const int64_t mr = m + r < m1 ? m + r : m;   // a missing row repeats the first one and is dropped below
-      slot[r] = members ? (int64_t)members[mr] : mr;
-      row[r] = reinterpret_cast<const uint4*>(slab + slot[r] * dim);
+      pos[r] = m + r < m1 ? m + r : m;   // a missing row repeats the first one and is dropped below
+      const int64_t at = (members && !sorted_rows) ? (int64_t)members[pos[r]] : pos[r];
+      row[r] = reinterpret_cast<const uint4*>(((members && sorted_rows) ? sorted_rows : slab) + at * dim);
       acc[r] = 0.0f;
     }
     for (int ch = lane; ch < n_chunks; ch += 32) {
@@ -338,8 +362,9 @@ cluster_scan_topk_kernel(const __nv_bfloat16* __restrict__ slab, int64_t n, int 
     }
 #pragma unroll
     for (int r = 0; r < CS_ROWS; ++r) {
-      if (m + r < m1) {   // warp-uniform
-        const uint64_t key = make_key(acc[r], (uint32_t)slot[r]);
+      if (m + r < m1 && score_to_ord(acc[r]) >= (uint32_t)(thr >> 32)) {   // warp-uniform (every lane holds the sum)
+        const int64_t slot = members ? (int64_t)members[pos[r]] : pos[r];
+        const uint64_t key = make_key(acc[r], (uint32_t)slot);
         if (key > thr) thr = warp_sorted_insert(my_list, k, key, lane);
       }
     }
@@ -353,7 +378,7 @@ cluster_scan_topk_kernel(const __nv_bfloat16* __restrict__ slab, int64_t n, int 
   }
 }
 
-cudaError_t launch_cluster_scan(const void* slab, int64_t n, int dim, const float* q_f32, int nq, int k,
+cudaError_t launch_cluster_scan(const void* slab, const void* sorted_rows, int64_t n, int dim, const float* q_f32, int nq, int k,
                                 const int64_t* probes, int n_probe, int n_split, int n_tail, const int* offsets,
                                 const int* order, int64_t n_indexed, uint64_t* partials, cudaStream_t st) {
   const int n_lists = n_probe * n_split + n_tail;
@@ -361,8 +386,8 @@ cudaError_t launch_cluster_scan(const void* slab, int64_t n, int dim, const floa
   const size_t smem = (size_t)dim * 4 + (size_t)CS_WARPS * k * 8;
   if (smem > 48 * 1024) return cudaErrorInvalidValue;
   return launch_overlapped(cluster_scan_topk_kernel, dim3((unsigned)(nq * n_lists)), dim3(CS_WARPS * 32), smem, st, 1,
-                           static_cast<const __nv_bfloat16*>(slab), n, dim, q_f32, nq, k, probes, n_probe, n_split,
-                           n_tail, offsets, order, n_indexed, partials);
+                           static_cast<const __nv_bfloat16*>(slab), static_cast<const __nv_bfloat16*>(sorted_rows), n, dim,
+                           q_f32, nq, k, probes, n_probe, n_split, n_tail, offsets, order, n_indexed, partials);
 }
 
 }  // namespace icc

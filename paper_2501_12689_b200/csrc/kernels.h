@@ -82,16 +82,18 @@ struct ScanParams {
 cudaError_t launch_scan(const ScanParams& p, cudaStream_t st);
 cudaError_t scan_configure(int smem_optin);
 
-// tcgen05 scoring: query tiles of 128 x row tiles of 256, top-k fused in the epilogue.
+// tcgen05 scoring: query tiles of 128 (or one resident tile of 64) x row tiles of 256, top-k fused
+// in the epilogue.
 struct UmmaParams {
-  CUtensorMap tmap_q;     // [nq_pad, dim] bf16, box 64 x 128, 128-byte swizzle
+  CUtensorMap tmap_q;     // [nq_pad, dim] bf16, box 64 x 128 (64 x 64 with q_resident), 128-byte swizzle
   CUtensorMap tmap_slab;  // [capacity, dim] bf16, box 64 x 256, 128-byte swizzle
-  CUtensorMap tmap_slab_half;  // same tensor, box 64 x 128 (CTA pairs: each CTA loads half a tile)
+  CUtensorMap tmap_slab_half;  // same tensor, box 64 x 128 (CTA pairs and resident queries)
   int cta_group;          // 1, or 2 = CTA pairs sharing each row tile
+  int q_resident;         // 1: at most 64 queries, M = 64, the query tile stays in shared memory
   int64_t n;
   int64_t tile_begin, tile_end;   // 256-row tiles scored by this launch
   int dim;
-  int q0, nq, k;          // queries [q0, q0 + n_query_tiles*128) of the staged batch
+  int nq, k;
   const uint64_t* thr_floor;      // optional [nq] keys: candidates at or below are discarded
   int n_query_tiles;
   int n_part;
@@ -100,13 +102,18 @@ struct UmmaParams {
   int smem_bytes;
   uint64_t* partials;     // [n_part][nq][k]
   unsigned long long* pace;   // optional [n_part][units per partition] progress words (L2 pacing hint)
-  unsigned pace_epoch;        // distinguishes this launch's progress words from older ones
+  unsigned epoch;             // number of this launch, unique in the process: tells this launch's progress
+                              // words and seeding flags from older ones
   int pace_window;            // tiles a CTA may run ahead of its slowest sibling
-  float* maxima_out;          // non-NULL: maxima-only launch over full tiles; receives
-                              // [tile - tile_begin][nq][4] group maxima, partials is not written
+  float* seed_maxima;         // optional [n_query_tiles][n_part][seed_t0][128][4]: seeding inside the launch (needs
+  unsigned* seed_flags;       // thr_floor == NULL and full first tiles); flags [n_query_tiles][n_part][4]
+  int seed_t0;                // tiles per CTA whose group maxima are exchanged (the first seed_t0 - 1 of them
+                              // are visited for their maxima only and scored at the end of the launch)
   int* dev_status;
 };
 cudaError_t launch_umma(const UmmaParams& p, cudaStream_t st);
+// Dynamic shared memory a launch of that shape needs.
+size_t umma_smem_bytes(int cta_group, bool q_resident, int dim, int k, int queue_cap, int n_stages);
 cudaError_t umma_configure(int smem_optin);
 
 // Merge n_part partial lists per query into the final sorted top-k and gather ids.  Entries
@@ -121,10 +128,6 @@ cudaError_t launch_merge(const uint64_t* partials, int n_part, int nq, int k, co
 // and out_thr [nq] = the k-th key (KEY_EMPTY when fewer than k candidates exist).
 cudaError_t launch_merge_keys(const uint64_t* partials, int n_part, int nq, int k, uint64_t* out_keys,
                               uint64_t* out_thr, cudaStream_t st);
-// Threshold from group maxima: maxima [n_tiles][nq][4] holds, per query, the best score of
-// n_tiles * 4 disjoint groups of cache rows; out_thr[q] becomes the key floor that admits every
-// score >= the k-th largest of them (KEY_EMPTY when there are fewer than k groups).
-cudaError_t launch_select_floor(const float* maxima, int n_tiles, int nq, int k, uint64_t* out_thr, cudaStream_t st);
 cudaError_t merge_configure(int smem_optin);
 
 // ---- two-level search (index_kernels.cu)
@@ -142,10 +145,14 @@ cudaError_t launch_sort_by_cluster(const int64_t* assign, int64_t n, int n_clust
 // Centroid c (row c of centroids, bf16) becomes the unit-length mean of its member rows.
 cudaError_t launch_centroid_update(const void* slab, int dim, const int* offsets, const int* order, int n_clusters,
                                    void* centroids, cudaStream_t st);
+// Row p of out_rows becomes cache row order[p] (the cluster-contiguous copy the two-level search streams).
+cudaError_t launch_gather_by_order(const void* slab, const int* order, int64_t n_rows, int dim, void* out_rows,
+                                   cudaStream_t st);
 // Scores, per query, the rows of its n_probe probed clusters (probes [nq][n_probe], -1 = none),
 // each cut into n_split pieces, and the rows [n_indexed, n) cut into n_tail pieces; writes one
 // sorted partial list per piece: partials [n_probe*n_split + n_tail][nq][k].
-cudaError_t launch_cluster_scan(const void* slab, int64_t n, int dim, const float* q_f32, int nq, int k,
+// sorted_rows (optional): rows of the indexed slots in member-list order (row p = cache row order[p]).
+cudaError_t launch_cluster_scan(const void* slab, const void* sorted_rows, int64_t n, int dim, const float* q_f32, int nq, int k,
                                 const int64_t* probes, int n_probe, int n_split, int n_tail, const int* offsets,
                                 const int* order, int64_t n_indexed, uint64_t* partials, cudaStream_t st);
 

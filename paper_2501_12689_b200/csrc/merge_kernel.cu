@@ -124,47 +124,6 @@ merge_topk_kernel(const uint64_t* __restrict__ partials, int n_part, int nq, int
   }
 }
 
-constexpr int SELECT_THREADS = 256;
-constexpr int SELECT_MAX_VALUES = 1280;
-
-// Per query: the k-th largest of m = n_tiles * 4 group maxima, by rank counting (m is a few
-// hundred).  CTA (q, c) ranks values c*256 .. c*256+255 of query q, one per thread, against a
-// shared copy of all m values held as unique 64-bit keys (score, then lower index first), so a
-// pair costs one integer compare.  Each maximum belongs to a different group of cache rows, so
-// k rows score at least the k-th largest value and it is a floor for the query's top-k.
-// Dependent kernels are released only at the end: a tensor-core CTA that starts early and waits
-// on the same SM was measured to slow this kernel's CTAs down several times over.
-__global__ void __launch_bounds__(SELECT_THREADS)
-select_floor_kernel(const float* __restrict__ maxima, int n_tiles, int nq, int k, uint64_t* __restrict__ out_thr) {
-  __shared__ uint64_t keys[SELECT_MAX_VALUES];
-  const int q = blockIdx.x, tid = threadIdx.x;
-  const int m = n_tiles * 4;
-  grid_dep_wait();   // the maxima come from the previous kernel
-  for (int t = tid; t < n_tiles; t += SELECT_THREADS) {
-    const float4 g = *reinterpret_cast<const float4*>(maxima + ((size_t)t * nq + q) * 4);
-    keys[4 * t] = make_key(g.x, (uint32_t)(4 * t));
-    keys[4 * t + 1] = make_key(g.y, (uint32_t)(4 * t + 1));
-    keys[4 * t + 2] = make_key(g.z, (uint32_t)(4 * t + 2));
-    keys[4 * t + 3] = make_key(g.w, (uint32_t)(4 * t + 3));
-  }
-  if (tid == 0 && blockIdx.y == 0 && m < k) out_thr[q] = KEY_EMPTY;
-  __syncthreads();
-  const int i = blockIdx.y * SELECT_THREADS + tid;
-  const uint64_t mine = i < m ? keys[i] : ~0ull;
-  int rank = 0;   // keys larger than mine
-#pragma unroll 8
-  for (int j = 0; j < m; ++j) rank += keys[j] > mine ? 1 : 0;
-  // admit every key whose score is >= this value: the smallest such key carries the largest slot word
-  if (i < m && rank == k - 1) out_thr[q] = (mine | 0xffffffffull) - 0xffffffffull - 1;
-  grid_dep_launch_dependents();
-}
-
-cudaError_t launch_select_floor(const float* maxima, int n_tiles, int nq, int k, uint64_t* out_thr, cudaStream_t st) {
-  if (n_tiles < 1 || n_tiles * 4 > SELECT_MAX_VALUES || !maxima || !out_thr) return cudaErrorInvalidValue;
-  const dim3 grid((unsigned)nq, (unsigned)((n_tiles * 4 + SELECT_THREADS - 1) / SELECT_THREADS));
-  return launch_overlapped(select_floor_kernel, grid, dim3(SELECT_THREADS), 0, st, 1, maxima, n_tiles, nq, k, out_thr);
-}
-
 static int g_merge_smem_limit = 48 * 1024;
 
 cudaError_t merge_configure(int smem_optin) {

@@ -54,25 +54,36 @@ def test_plan_paths_and_shapes():
     p = pkg.ic_cache_plan(1024, 4_000_000, 256, 32)
     assert p["n_query_tiles"] == 2 and p["n_partitions"] == 74 and p["n_ctas"] == 148
     p = pkg.ic_cache_plan(768, 16_000_000, 1024, 64)
-    assert p["n_query_tiles"] == 8 and p["n_partitions"] == 18 and p["n_ctas"] == 144 and p["n_launches"] == 3
-    assert p["cta_group"] == 2 and 0 < p["seed0_tiles"] < p["seed_tiles"] and p["seed0_tiles"] % 18 == 0
+    assert p["n_query_tiles"] == 8 and p["n_partitions"] == 18 and p["n_ctas"] == 144 and p["n_launches"] == 2
+    assert p["cta_group"] == 2 and p["seed0_tiles"] == 162 < p["seed_tiles"] and p["query_resident"] == 0   # 9 tiles for each of 18 partitions
     assert p["smem_bytes"] <= 232448
     assert p["seed_tiles"] > 0 and p["seed_tiles"] % 18 == 0 and p["seed_tiles"] * 256 * 15 < 16_000_000
     assert pkg.ic_cache_plan(768, 70_001, 64, 10)["seed_tiles"] == 0      # too few tiles per CTA
     assert pkg.ic_cache_plan(768, 70_001, 64, 10)["seed0_tiles"] == 0
-    # threshold seeding: a maxima-only launch over about one tile per SM; a list-level sample of
-    # 1/16 of the tiles only on large caches; neither for a handful of queries with short lists
+    # threshold seeding: inside the scoring launch, from the first tile of every partition; a
+    # list-level sample of 1/16 of the tiles, in a launch of its own, only on large caches
     p = pkg.ic_cache_plan(768, 1_000_000, 64, 10)
-    assert (p["seed0_tiles"], p["seed_tiles"]) == (148, 0)
+    assert (p["seed0_tiles"], p["seed_tiles"], p["n_launches"]) == (148, 0, 1)
     p = pkg.ic_cache_plan(768, 16_000_000, 64, 64)
     assert p["seed0_tiles"] == 148 and p["seed_tiles"] == 16_000_000 // 256 // 16 // 148 * 148
     p = pkg.ic_cache_plan(1024, 4_000_000, 256, 32)
     assert p["seed0_tiles"] == 148 and p["seed_tiles"] % 74 == 0 and p["seed_tiles"] > 148
-    assert pkg.ic_cache_plan(768, 16_000_000, 1024, 64)["seed0_tiles"] == 162          # 9 tiles for each of 18 partitions
-    for nq, k, seeded in ((8, 10, False), (8, 16, False), (9, 10, True), (8, 17, True), (4, 64, True)):
-        assert (pkg.ic_cache_plan(768, 1_000_000, nq, k, path=pkg.IC_PATH_UMMA)["seed0_tiles"] > 0) == seeded
+    # the exchanged sample stays at about one tile per SM however few partitions there are
+    assert pkg.ic_cache_plan(768, 40_000, 1024, 128)["seed0_tiles"] == 144      # 8 tiles for each of 18 partitions
+    # batches of at most 64 queries keep the query tile in shared memory (M = 64) while a ring of
+    # four 16 KiB stages still fits beside it
+    p = pkg.ic_cache_plan(768, 1_000_000, 64, 10)
+    assert p["query_resident"] == 1 and p["query_tile"] == 64 and p["n_stages"] >= 6 and p["smem_bytes"] <= 232448
+    assert pkg.ic_cache_plan(768, 1_000_000, 65, 10)["query_resident"] == 0
+    assert pkg.ic_cache_plan(768, 16_000_000, 64, 64)["query_resident"] == 1
+    assert pkg.ic_cache_plan(2048, 1_000_000, 8, 10)["query_resident"] == 0      # 256 KiB of queries do not fit
+    for dim in (8, 384, 768, 1024, 1536, 4096):
+        for nq in (1, 64, 128, 1024):
+            for k in (1, 10, 64, 128):
+                p = pkg.ic_cache_plan(dim, 1_000_000, nq, k, path=pkg.IC_PATH_UMMA)
+                assert p["smem_bytes"] <= 232448 and p["n_stages"] >= 2 and p["queue_cap"] >= 1
     p = pkg.ic_cache_plan(768, 16_000_000, 3000, 64)
-    assert p["n_launches"] == 9
+    assert p["n_launches"] == 6
     assert pkg.ic_cache_plan(768, 1_000_000, 300, 10)["cta_group"] == 1    # odd number of query tiles
     p = pkg.ic_cache_plan(2048, 1000, 2, 5)          # too wide for the scan path
     assert p["path"] == pkg.IC_PATH_UMMA
