@@ -47,7 +47,14 @@ NOMINAL_BF16_TFLOPS = 2250.0
 # captures run on a scaled-down cache, and the traffic of this kernel grows in proportion to the
 # rows scanned.  Key: (kernel, dim).  An entry is removed (the line then says null) whenever that
 # kernel changes after its capture.
-NCU_TRAFFIC_BYTES_PER_ROW = {}
+NCU_TRAFFIC_BYTES_PER_ROW = {
+    # profiles/umma_stress_2m_q1024.md: main pass, CTA pairs, 2,891,083,776 B over 1,877,632 scanned rows
+    ("umma_score_topk_kernel<2,streamed> (main pass)", 768): 2_891_083_776 / 1_877_632,
+    # profiles/umma_dense_1m_q256.md: CTA pairs, 2,094,998,016 B over 1,000,512 rows (incl. the re-read first tiles)
+    ("umma_score_topk_kernel<2,streamed> (main pass)", 1024): 2_094_998_016 / 1_000_512,
+    # profiles/umma_online_q64.md: resident query tile, 1,542,186,496 B over 1,000,128 rows
+    ("umma_score_topk_kernel<1,resident> (main pass)", 768): 1_542_186_496 / 1_000_128,
+}
 
 
 def parse_args():
@@ -69,11 +76,14 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--minimal", action="store_true",
                     help="headline measurement only (profiling aid): implies every --no-* switch")
+    ap.add_argument("--only-widening", action="store_true",
+                    help="with --minimal: keep the widening workload of the chosen configuration (profiling aid)")
     ap.add_argument("--two-level-nprobe", type=int, default=4)
     ap.add_argument("--self-similarity-rows", type=int, default=65536)
     a = ap.parse_args()
     if a.minimal:
-        a.no_sweep = a.no_crossover = a.no_configs = a.no_widening = a.no_cpu_baseline = a.no_e2e = True
+        a.no_sweep = a.no_crossover = a.no_configs = a.no_cpu_baseline = a.no_e2e = True
+        a.no_widening = not a.only_widening
     return a
 
 
@@ -353,7 +363,8 @@ class Bench:
             out = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                    "frac": ach / peaks["bf16_tflops_sustained"], "frac_of_nominal": ach / NOMINAL_BF16_TFLOPS,
                    "frac_of_burst_peak": ach / peaks["bf16_tflops"]}
-        kernel = {2: "scan_score_topk_kernel", 3: "umma_score_topk_kernel (main pass)",
+        variant = "<1,resident>" if pl["query_resident"] else f"<{pl['cta_group']},streamed>"
+        kernel = {2: "scan_score_topk_kernel", 3: f"umma_score_topk_kernel{variant} (main pass)",
                   1: "generic_score_topk_kernel"}[pl["path"]]
         per_row = NCU_TRAFFIC_BYTES_PER_ROW.get((kernel, w.dim))
         out.update({"traffic": per_row * rows_main if per_row else None,
@@ -502,10 +513,14 @@ def run_ours(args):
             crossover.append((name, b.measure(q, repeats=3, steps=min(steps, 5), warmup=3, forced_path=code)))
     plan = ic_cache_plan(w.dim, w.n, nq, w.k, b.path, props.multi_processor_count, props.shared_memory_per_block_optin)
     n_start = b.n0
+    others, two_level, self_sim = [], None, None
+    if not args.no_widening and w.name == "clustered":
+        two_level = run_widening_two_level(b, args.two_level_nprobe)
+    if not args.no_widening and w.name == "online":
+        self_sim = run_widening_self_similarity(b, args.self_similarity_rows)
     b.close()
 
     # ---- the other configurations, compactly, and the two widening workloads
-    others, two_level, self_sim = [], None, None
     if not args.no_configs or not args.no_widening:
         for name in ("online", "clustered", "dense"):
             if name == w.name:
