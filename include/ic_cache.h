@@ -293,7 +293,10 @@ int ic_cache_utility_read(ic_cache_t* c, int64_t* ids_host, float* utility_host)
  * else 1 .. min(size, IC_MAX_CLUSTERS).  n_iters >= 0 update steps (0 keeps the initial
  * centroids).  init_slots_host: HOST array of n_clusters distinct slots whose rows are the
  * initial centroids, or NULL for slots floor(c * size / n_clusters).  Entries are not moved:
- * slots, ids and the results of ic_cache_query are unaffected.  Not part of the per-request
+ * slots, ids and the results of ic_cache_query are unaffected.  The index keeps its own copy of the
+ * indexed rows in cluster order (size * dim * 2 bytes more device memory) so that a probed cluster
+ * is one contiguous run to read; if that allocation fails the search reads rows through the member
+ * lists instead (slower, same results).  Not part of the per-request
  * path (each iteration scores every entry against every centroid and reads the slab once
  * more); synchronises the stream.  Replaces any earlier index.  ic_cache_remove and
  * ic_cache_clear drop the index; entries inserted later stay outside it and are searched

@@ -1442,6 +1442,19 @@ int ic_cache_query_clustered(ic_cache_t* c, const void* q, int32_t nq, int32_t k
     const int64_t avg_cluster = std::max<int64_t>(1, c->n_indexed / c->n_clusters);
     int n_split = (int)std::max<int64_t>(1, std::min<int64_t>({16, (6 * c->sm_count + (int64_t)w * np - 1) / ((int64_t)w * np),
                                                                 avg_cluster / 64}));
+    // Streaming the probed clusters from the cluster-contiguous copy pays from a few dozen (query,
+    // probe) pairs on: pieces of at least ~256 rows, two CTAs per SM.
+    int stream_split = 0, stream_stages = 0;
+    if (c->have_idx_rows && c->dim <= 1024 && (int64_t)w * np >= 32) {
+      // about four waves of CTAs (two per SM), so that the last wave's idle SMs cost little
+      stream_split = (int)std::max<int64_t>(1, std::min<int64_t>({16, (8 * c->sm_count + (int64_t)w * np - 1) / ((int64_t)w * np),
+                                                                   avg_cluster / 256}));
+      const int half = c->smem_optin / 2 - 2048;
+      stream_stages = 2;
+      while (stream_stages < 4 && icc::cluster_stream_smem_bytes(c->dim, k, stream_stages + 1) <= half) ++stream_stages;
+      if (icc::cluster_stream_smem_bytes(c->dim, k, stream_stages) > c->smem_optin) stream_split = 0;
+      else n_split = stream_split;
+    }
     // Rows inserted since the build are one contiguous range that every query scans: from a
     // thousand rows on, the tiles that lie wholly past the index go to the tensor-core kernel (one
     // launch over that tile range, its per-CTA lists joining the final merge; measured with
@@ -1478,11 +1491,34 @@ int ic_cache_query_clustered(ic_cache_t* c, const void* q, int32_t nq, int32_t k
     // the same bf16-rounded queries, widened to fp32, for the scan of the clusters
     cudaError_t e = icc::launch_convert_rows(qw, c->input_dtype == IC_F32, w, c->dim, c->normalize, c->q_bf16.p,
                                              static_cast<float*>(c->q_f32.p), nq_pad, nullptr, nullptr, c->stream);
+    // The probed clusters: with the cluster-contiguous copy and enough (query, probe) pairs to fill
+    // the GPU, one bulk-copy pipeline per piece (two CTAs per SM); otherwise the register-load kernel,
+    // which also takes the ragged rows past the index.
+    const bool stream = c->have_idx_rows && c->dim <= 1024 && stream_split > 0;
+    if (e == cudaSuccess && stream) {
+      icc::ClusterStreamParams cp;
+      cp.sorted_rows = c->idx_rows.p;
+      cp.dim = c->dim;
+      cp.q_f32 = static_cast<const float*>(c->q_f32.p);
+      cp.nq = w;
+      cp.k = k;
+      cp.probes = probes;
+      cp.n_probe = nprobe;
+      cp.n_split = n_split;
+      cp.offsets = static_cast<const int*>(c->idx_offsets.p);
+      cp.order = static_cast<const int*>(c->idx_order.p);
+      cp.partials = static_cast<uint64_t*>(c->partials.p);
+      cp.n_stages = stream_stages;
+      cp.smem_bytes = icc::cluster_stream_smem_bytes(c->dim, k, stream_stages);
+      cp.dev_status = c->d_status;
+      e = icc::launch_cluster_stream(cp, c->stream);
+      c->launches += 1;
+    }
     if (e == cudaSuccess)
-      e = icc::launch_cluster_scan(c->slab, c->have_idx_rows ? c->idx_rows.p : nullptr, scan_end, c->dim, static_cast<const float*>(c->q_f32.p), w, k, probes, nprobe,
-                                   n_split, n_tail, static_cast<const int*>(c->idx_offsets.p),
-                                   static_cast<const int*>(c->idx_order.p), c->n_indexed,
-                                   static_cast<uint64_t*>(c->partials.p), c->stream);
+      e = icc::launch_cluster_scan(c->slab, c->have_idx_rows ? c->idx_rows.p : nullptr, scan_end, c->dim,
+                                   static_cast<const float*>(c->q_f32.p), w, k, probes, nprobe, n_split, n_tail,
+                                   static_cast<const int*>(c->idx_offsets.p), static_cast<const int*>(c->idx_order.p),
+                                   c->n_indexed, static_cast<uint64_t*>(c->partials.p), stream ? np * n_split : 0, c->stream);
     if (e != cudaSuccess) return fail(IC_ERR_CUDA, "two-level search launch failed: %s", cudaGetErrorString(e));
     if (dense_tail) {
       int unused = 0;

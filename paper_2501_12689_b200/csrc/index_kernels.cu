@@ -284,14 +284,15 @@ __global__ void __launch_bounds__(CS_WARPS * 32)
 cluster_scan_topk_kernel(const __nv_bfloat16* __restrict__ slab, const __nv_bfloat16* __restrict__ sorted_rows, int64_t n,
                          int dim, const float* __restrict__ q_f32, int nq, int k, const int64_t* __restrict__ probes,
                          int n_probe, int n_split, int n_tail, const int* __restrict__ offsets,
-                         const int* __restrict__ order, int64_t n_indexed, uint64_t* __restrict__ partials) {
+                         const int* __restrict__ order, int64_t n_indexed, uint64_t* __restrict__ partials, int l_begin) {
   extern __shared__ __align__(16) unsigned char cs_smem[];
   float* qs = reinterpret_cast<float*>(cs_smem);                         // [dim]
   uint64_t* lists = reinterpret_cast<uint64_t*>(qs + dim);               // [CS_WARPS][k]
   __shared__ uint64_t win_key[MAX_K];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_lists = n_probe * n_split + n_tail;
-  const int q = blockIdx.x / n_lists, l = blockIdx.x - q * n_lists;
+  const int lists_here = n_lists - l_begin;
+  const int q = blockIdx.x / lists_here, l = l_begin + (blockIdx.x - q * lists_here);
   grid_dep_launch_dependents();
   grid_dep_wait();   // probes and the prepared query come from earlier kernels in the stream
   for (int j = tid; j < dim; j += CS_WARPS * 32) qs[j] = q_f32[(size_t)q * dim + j];
@@ -380,14 +381,15 @@ cluster_scan_topk_kernel(const __nv_bfloat16* __restrict__ slab, const __nv_bflo
 
 cudaError_t launch_cluster_scan(const void* slab, const void* sorted_rows, int64_t n, int dim, const float* q_f32, int nq, int k,
                                 const int64_t* probes, int n_probe, int n_split, int n_tail, const int* offsets,
-                                const int* order, int64_t n_indexed, uint64_t* partials, cudaStream_t st) {
+                                const int* order, int64_t n_indexed, uint64_t* partials, int l_begin, cudaStream_t st) {
   const int n_lists = n_probe * n_split + n_tail;
-  if (nq <= 0 || n_lists <= 0) return cudaErrorInvalidValue;
+  if (nq <= 0 || n_lists <= 0 || l_begin < 0 || l_begin > n_lists) return cudaErrorInvalidValue;
+  if (l_begin == n_lists) return cudaSuccess;   // nothing left for this kernel
   const size_t smem = (size_t)dim * 4 + (size_t)CS_WARPS * k * 8;
   if (smem > 48 * 1024) return cudaErrorInvalidValue;
-  return launch_overlapped(cluster_scan_topk_kernel, dim3((unsigned)(nq * n_lists)), dim3(CS_WARPS * 32), smem, st, 1,
+  return launch_overlapped(cluster_scan_topk_kernel, dim3((unsigned)(nq * (n_lists - l_begin))), dim3(CS_WARPS * 32), smem, st, 1,
                            static_cast<const __nv_bfloat16*>(slab), static_cast<const __nv_bfloat16*>(sorted_rows), n, dim,
-                           q_f32, nq, k, probes, n_probe, n_split, n_tail, offsets, order, n_indexed, partials);
+                           q_f32, nq, k, probes, n_probe, n_split, n_tail, offsets, order, n_indexed, partials, l_begin);
 }
 
 }  // namespace icc

@@ -130,6 +130,25 @@ cudaError_t launch_merge_keys(const uint64_t* partials, int n_part, int nq, int 
                               uint64_t* out_thr, cudaStream_t st);
 cudaError_t merge_configure(int smem_optin);
 
+// Two-level search, pieces of probed clusters streamed from the cluster-contiguous copy of the rows
+// (scan_kernel.cu; dim <= 1024).  One CTA per (query, probe, piece); partials as for launch_cluster_scan.
+struct ClusterStreamParams {
+  const void* sorted_rows;   // row p = cache row order[p]
+  int dim;
+  const float* q_f32;
+  int nq, k;
+  const int64_t* probes;     // [nq][n_probe], -1 = none
+  int n_probe, n_split;
+  const int* offsets;
+  const int* order;
+  uint64_t* partials;        // [n_probe * n_split (+ lists of other kernels)][nq][k]
+  int n_stages;
+  int smem_bytes;
+  int* dev_status;
+};
+cudaError_t launch_cluster_stream(const ClusterStreamParams& p, cudaStream_t st);
+int cluster_stream_smem_bytes(int dim, int k, int n_stages);
+
 // ---- two-level search (index_kernels.cu)
 constexpr int IC_INDEX_MAX_CLUSTERS = 16384;   // must equal IC_MAX_CLUSTERS; bounds the sort kernels' shared memory
 cudaError_t index_configure(int smem_optin);
@@ -152,8 +171,9 @@ cudaError_t launch_gather_by_order(const void* slab, const int* order, int64_t n
 // each cut into n_split pieces, and the rows [n_indexed, n) cut into n_tail pieces; writes one
 // sorted partial list per piece: partials [n_probe*n_split + n_tail][nq][k].
 // sorted_rows (optional): rows of the indexed slots in member-list order (row p = cache row order[p]).
+// l_begin: first list this launch produces (n_probe * n_split when another kernel scans the clusters).
 cudaError_t launch_cluster_scan(const void* slab, const void* sorted_rows, int64_t n, int dim, const float* q_f32, int nq, int k,
                                 const int64_t* probes, int n_probe, int n_split, int n_tail, const int* offsets,
-                                const int* order, int64_t n_indexed, uint64_t* partials, cudaStream_t st);
+                                const int* order, int64_t n_indexed, uint64_t* partials, int l_begin, cudaStream_t st);
 
 }  // namespace icc

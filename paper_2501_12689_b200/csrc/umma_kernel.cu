@@ -22,11 +22,13 @@
 //   <1, true>   at most 64 queries: M = 64, the whole query tile is loaded once and stays in
 //               shared memory, ring stages hold 128 cache rows (16 KiB) and nothing else
 //
-// Threshold seeding inside the launch: every CTA first reads its first accumulator only for the
-// maxima of four groups of 64 rows per query and publishes them; once the CTAs that score the
-// same queries have all published (a bounded look, never a condition for progress), each epilogue
-// thread takes the k-th largest of those maxima as the floor of its query: k different rows score
-// at least that much, so nothing below it can be in the top-k.
+// Threshold seeding inside the launch: every CTA first visits its first few tiles only for the
+// maxima of four groups of 64 rows per query (the last of them with the accumulator held back)
+// and publishes them; once the CTAs that score the same queries have all published (a bounded
+// look, never a condition for progress), each epilogue thread folds all those maxima into bins of
+// disjoint rows and takes a score that at least k bins reach as the floor of its query: k
+// different rows score at least that much, so nothing below it can be in the top-k.  The tiles
+// visited for their maxima only are scored at the end of the CTA's tile sequence.
 #include <math.h>
 #include <string.h>
 

@@ -115,7 +115,7 @@ def test_threshold_seeding_pass(order, nq, k):
 
 @pytest.mark.parametrize("order", ["random", "best_first", "best_last"])
 def test_two_level_threshold_seeding(order):
-    # enough tiles that a sample of them is scored into lists between the maxima launch and the main pass
+    # enough tiles that a sample of them is scored into lists, by a launch of its own, ahead of the main pass
     _seeding_case(order, 40, 16, 2_600_011, levels=2)
 
 
@@ -126,7 +126,7 @@ def _seeding_case(order, nq, k, n, levels):
     from paper_2501_12689_b200 import ic_cache_plan
     dim = 64
     plan = ic_cache_plan(dim, n, nq, k, IC_PATH_UMMA)
-    # level 0: maxima-only launch (its tiles are scored again); level 1: a sample scored into lists
+    # level 0: group maxima exchanged inside the scoring launch; level 1: a sample scored into lists
     assert plan["seed0_tiles"] > 0 and (plan["seed_tiles"] > 0) == (levels == 2)
     x, q = _gauss(n, dim, nq, seed=55)
     if order != "random":
