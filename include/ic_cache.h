@@ -351,7 +351,10 @@ int64_t ic_cache_size(const ic_cache_t* c);
 int ic_cache_clear(ic_cache_t* c);
 
 /* Synchronise the handle's stream and report IC_ERR_TIMEOUT if any kernel since the last
- * call of this function gave up on a bounded wait, IC_ERR_CUDA on a CUDA error, else IC_OK. */
+ * call of this function gave up on a bounded wait, IC_ERR_CUDA on a CUDA error, else IC_OK.
+ * (The debug build of the library, libic_cache_debug.so, compiled with -DIC_CACHE_DEBUG_CHECKS,
+ * additionally checks tile, list and slot indices on the device; a failed check is reported here
+ * the same way, with a message that says so.  No build ever traps on the device.) */
 int ic_cache_sync(ic_cache_t* c);
 
 /*

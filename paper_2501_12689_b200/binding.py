@@ -15,7 +15,9 @@ from typing import Optional, Tuple
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libic_cache.so")
+# IC_CACHE_LIB names another build of the same library (the debug build with index checks,
+# libic_cache_debug.so); there is still no fallback if it is missing
+LIB_PATH = os.environ.get("IC_CACHE_LIB") or os.path.join(_PKG, "libic_cache.so")
 
 IC_OK, IC_ERR_INVALID, IC_ERR_NOMEM, IC_ERR_FULL = 0, -1, -2, -3
 IC_ERR_CUDA, IC_ERR_UNSUPPORTED, IC_ERR_TIMEOUT = -4, -5, -6

@@ -11,7 +11,7 @@ constexpr unsigned FULL_MASK = 0xffffffffu;
 constexpr uint64_t KEY_EMPTY = 0ull;  // smaller than every real key
 
 // Status word values written by kernels whose bounded waits expire (device -> host).
-enum : int { DEV_OK = 0, DEV_TIMEOUT_LOCK = 1, DEV_TIMEOUT_MBAR = 2 };
+enum : int { DEV_OK = 0, DEV_TIMEOUT_LOCK = 1, DEV_TIMEOUT_MBAR = 2, DEV_CHECK_FAILED = 3 };
 
 // Monotone map from fp32 scores to unsigned integers (-0 is folded onto +0 first so that
 // equal scores give equal keys).
@@ -40,6 +40,20 @@ __device__ __forceinline__ void report_status(int* dev_status, int code) {
   *reinterpret_cast<volatile int*>(dev_status) = code;
   __threadfence_system();
 }
+
+// Index checks of the debug build (-DIC_CACHE_DEBUG_CHECKS, libic_cache_debug.so): a failed check
+// writes DEV_CHECK_FAILED to the status word, which the host reports like an expired wait; it never
+// traps.  In the normal build the macro is empty.
+#ifdef IC_CACHE_DEBUG_CHECKS
+#define ICC_CHECK(cond, dev_status)                                        \
+  do {                                                                     \
+    if (!(cond)) icc::report_status((dev_status), icc::DEV_CHECK_FAILED);  \
+  } while (0)
+#else
+#define ICC_CHECK(cond, dev_status) \
+  do {                              \
+  } while (0)
+#endif
 
 // Insert `key` into a descending list of k entries in shared memory, dropping the last one.
 // All 32 lanes of the warp call this with the same arguments; the caller guarantees that no

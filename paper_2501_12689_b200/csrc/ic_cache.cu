@@ -309,7 +309,8 @@ void profile_mark(ic_cache* c, std::vector<cudaEvent_t>& pool, size_t& used) {
 
 int check_timeout(ic_cache* c) {
   if (c->h_status && *reinterpret_cast<volatile int*>(c->h_status) != 0)
-    return fail(IC_ERR_TIMEOUT, "an earlier kernel gave up on a bounded wait (code %d); call ic_cache_sync to clear", *c->h_status);
+    return fail(IC_ERR_TIMEOUT, *c->h_status == 3 ? "an earlier kernel failed a debug-build index check (code %d); call ic_cache_sync to clear"
+                                                  : "an earlier kernel gave up on a bounded wait (code %d); call ic_cache_sync to clear", *c->h_status);
   return IC_OK;
 }
 
@@ -1580,7 +1581,8 @@ int ic_cache_sync(ic_cache_t* c) {
   if (c->h_status && *reinterpret_cast<volatile int*>(c->h_status) != 0) {
     const int code = *c->h_status;
     *c->h_status = 0;
-    return fail(IC_ERR_TIMEOUT, "a kernel gave up on a bounded wait (code %d); its results are incomplete", code);
+    return fail(IC_ERR_TIMEOUT, code == 3 ? "a kernel failed a debug-build index check (code %d); its results are suspect"
+                                          : "a kernel gave up on a bounded wait (code %d); its results are incomplete", code);
   }
   return IC_OK;
 }

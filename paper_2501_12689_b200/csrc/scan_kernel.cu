@@ -168,6 +168,7 @@ scan_score_topk_kernel(const __nv_bfloat16* __restrict__ slab, int64_t n, int di
       const float score = transpose_reduce<V>(acc, lane);
       const int64_t row = piece * SCAN_STAGE_ROWS + warp * SCAN_ROWS_PER_WARP + my_row;
       const uint64_t key = make_key(score, (uint32_t)row);
+      ICC_CHECK(my_q < QB && piece < n_pieces, dev_status);
       const bool hit = reporter && row < n && key > thr;
       unsigned hits = __ballot_sync(FULL_MASK, hit);
       while (hits) {
@@ -319,6 +320,7 @@ cluster_stream_topk_kernel(const __nv_bfloat16* __restrict__ sorted_rows, int di
       // list's last score cannot enter
       const bool maybe = reporter && pos < m1 && score_to_ord(score) >= (uint32_t)(thr >> 32) && score == score;
       uint64_t key = KEY_EMPTY;
+      ICC_CHECK(!maybe || (pos >= m0 && pos < m1), dev_status);
       if (maybe) key = make_key(score, (uint32_t)order[pos]);
       unsigned hits = __ballot_sync(FULL_MASK, maybe && key > thr);
       while (hits) {

@@ -467,6 +467,7 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     bool ok = true;
     for (; lt < n_seq; ++lt) {
       const int64_t tile = tile_of(lt);
+      ICC_CHECK(tile >= tile_begin && tile < tile_end && cnt >= 0 && cnt <= qcap, dev_status);
       const int buf = (int)(lt & 1);
       const uint32_t bph = (uint32_t)((lt >> 1) & 1);
       ok = mbar_wait(&tail->acc_full[buf], bph, abort_flag);
@@ -716,9 +717,14 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     const int q_live = min(LW, nq - q_first);
     if (q_live > 0) {
       uint64_t* dst = partials + ((size_t)part * nq + q_first) * k;
+      ICC_CHECK(part < n_part && q_first + q_live <= nq, dev_status);
       for (int i = lane; i < q_live * k; i += 32) {
         const int ql = i / k, e = i - ql * k;
-        dst[i] = warp_lists[e * LW + ql];
+        const uint64_t key = warp_lists[e * LW + ql];
+        // a list holds real rows only, best first
+        ICC_CHECK(key == KEY_EMPTY || (int64_t)key_slot(key) < n, dev_status);
+        ICC_CHECK(e == 0 || key <= warp_lists[(e - 1) * LW + ql], dev_status);
+        dst[i] = key;
       }
     }
   }

@@ -33,6 +33,16 @@ def test_library_exports_every_declared_symbol():
     assert lib.ic_cache_version() >= 100
 
 
+def test_debug_build_exports_the_same_symbols():
+    """The debug build (index checks compiled in) is the same ABI: it builds without a GPU and
+    exports every declared symbol."""
+    import ctypes
+    from paper_2501_12689_b200.build import build
+    lib = ctypes.CDLL(build(debug_checks=True))
+    for name in _declared_symbols():
+        assert hasattr(lib, name), f"{name} is missing from the debug build"
+
+
 def test_header_constants_match_binding():
     text = open(os.path.join(ROOT, "include", "ic_cache.h")).read()
     assert int(re.search(r"#define IC_MAX_K (\d+)", text).group(1)) == binding.IC_MAX_K
