@@ -380,6 +380,11 @@ int run_umma_passes(ic_cache* c, const ic_cache_plan_t& pl, const void* q_bf16, 
   up.smem_bytes = pl.smem_bytes;
   up.dev_status = c->d_status;
   up.seed_t0 = pl.seed0_tiles / P;
+  up.seed_look_cycles = 60000;   // ~30 us
+  if (const char* env = getenv("IC_CACHE_SEED_LOOK_CYCLES")) {   // tuning and test knob: 0 = never wait for the siblings
+    const int v = atoi(env);
+    if (v >= 0) up.seed_look_cycles = v;
+  }
   // CTAs of one partition may run an eighth of the partition's share of L2 apart (measured: with
   // 18 partitions of 393 KB tiles, 3 tiles keep DRAM reads at the slab size, 8 tiles do not)
   up.pace = pace;

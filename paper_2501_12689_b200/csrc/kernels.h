@@ -107,6 +107,7 @@ struct UmmaParams {
   int pace_window;            // tiles a CTA may run ahead of its slowest sibling
   float* seed_maxima;         // optional [n_query_tiles][n_part][seed_t0][128][4]: seeding inside the launch (needs
   unsigned* seed_flags;       // thr_floor == NULL and full first tiles); flags [n_query_tiles][n_part][4]
+  int seed_look_cycles;       // longest an epilogue warp looks for its siblings' maxima, in SM cycles
   int seed_t0;                // tiles per CTA whose group maxima are exchanged (the first seed_t0 - 1 of them
                               // are visited for their maxima only and scored at the end of the launch)
   int* dev_status;

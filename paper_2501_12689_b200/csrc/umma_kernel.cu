@@ -54,7 +54,6 @@ constexpr int UM_MAX_STAGES = 12;
 constexpr int UM_TMEM_COLS = 512;
 constexpr int UM_CHUNK = 64;          // accumulator columns per epilogue step
 constexpr long long PACE_LIMIT_CYCLES = 100000;   // ~50 us: longest a CTA holds back for a slower sibling
-constexpr long long SEED_LOOK_LIMIT_CYCLES = 60000;   // ~30 us: longest an epilogue warp looks for its siblings' maxima
 constexpr uint32_t NAN_BITS = 0x7fc00000u;
 
 struct UmmaSmemTail {
@@ -183,7 +182,7 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                        int64_t n, int64_t tile_begin, int64_t tile_end, int dim, int nq, int k, int n_query_tiles,
                        int n_part, int n_stages, int qcap, const uint64_t* __restrict__ thr_floor_in,
                        uint64_t* __restrict__ partials, unsigned long long* pace, unsigned epoch, int pace_window,
-                       float* seed_maxima, unsigned* seed_flags, int seed_t0, int* dev_status) {
+                       float* seed_maxima, unsigned* seed_flags, int seed_t0, int seed_look_cycles, int* dev_status) {
   static_assert(!(QRES && CG == 2), "resident queries run on single CTAs");
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -534,7 +533,7 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             bool all = true;
             for (int p = lane; p < n_part; p += 32) all = all && (ld_acquire_gpu(fl + p * 4) == epoch);
             complete = __all_sync(FULL_MASK, all);
-            if (complete || __any_sync(FULL_MASK, clock64() - t0 > SEED_LOOK_LIMIT_CYCLES)) break;
+            if (complete || __any_sync(FULL_MASK, clock64() - t0 > (long long)seed_look_cycles)) break;
             __nanosleep(256);
           }
           const int n_ent = n_part * seed_t0;          // float4 entries per query: 4 * n_ent group maxima
@@ -763,7 +762,7 @@ static cudaError_t launch_umma_variant(const UmmaParams& p, cudaStream_t st) {
   return launch_overlapped(umma_score_topk_kernel<CG, QRES>, grid, dim3(UM_THREADS), (size_t)p.smem_bytes, st, CG, p.tmap_q,
                            slab_map, p.n, p.tile_begin, p.tile_end, p.dim, p.nq, p.k, p.n_query_tiles, p.n_part,
                            p.n_stages, p.queue_cap, p.thr_floor, p.partials, p.pace, p.epoch, p.pace_window,
-                           p.seed_maxima, p.seed_flags, p.seed_t0, p.dev_status);
+                           p.seed_maxima, p.seed_flags, p.seed_t0, p.seed_look_cycles, p.dev_status);
 }
 
 cudaError_t launch_umma(const UmmaParams& p, cudaStream_t st) {
@@ -777,7 +776,7 @@ cudaError_t launch_umma(const UmmaParams& p, cudaStream_t st) {
   if ((p.seed_maxima == nullptr) != (p.seed_flags == nullptr)) return cudaErrorInvalidValue;
   // seeding inside the launch reads the first seed_t0 tiles of every CTA as full tiles
   if (p.seed_maxima != nullptr &&
-      (p.seed_t0 < 1 || p.tile_end - p.tile_begin < (int64_t)p.n_part * p.seed_t0 ||
+      (p.seed_t0 < 1 || p.seed_look_cycles < 0 || p.tile_end - p.tile_begin < (int64_t)p.n_part * p.seed_t0 ||
        (p.tile_begin + (int64_t)p.n_part * p.seed_t0) * UM_RT > p.n))
     return cudaErrorInvalidValue;
   if (p.q_resident) return launch_umma_variant<1, true>(p, st);

@@ -119,6 +119,15 @@ def test_two_level_threshold_seeding(order):
     _seeding_case(order, 40, 16, 2_600_011, levels=2)
 
 
+@pytest.mark.parametrize("nq,k", [(40, 10), (130, 64)])
+def test_seeding_falls_back_to_local_floors_when_the_siblings_are_not_waited_for(nq, k, monkeypatch):
+    """The exchange of group maxima inside a launch is a bounded look, never a condition for
+    progress.  With the look cut to nothing, CTAs that do not find all their siblings' maxima at the
+    first glance score their first tile with a local floor instead: the results must not change."""
+    monkeypatch.setenv("IC_CACHE_SEED_LOOK_CYCLES", "0")
+    _seeding_case("random", nq, k, 400_003, levels=1)
+
+
 def _seeding_case(order, nq, k, n, levels):
     # enough row tiles per CTA that the tensor-core path takes a floor from a sample first and
     # starts the main pass from it; with the best rows all inside (or all outside) the sample,
