@@ -54,6 +54,8 @@ NCU_TRAFFIC_BYTES_PER_ROW = {
     ("umma_score_topk_kernel<2,streamed> (main pass)", 1024): 2_095_134_464 / 1_000_512,
     # profiles/umma_online_q64.md: resident query tile, 1,541,755,136 B over 1,000,128 rows
     ("umma_score_topk_kernel<1,resident> (main pass)", 768): 1_541_755_136 / 1_000_128,
+    # profiles/scan_online_q1.md: CUDA-core scan, 1,540,525,312 B over 1,000,002 rows
+    ("scan_score_topk_kernel", 768): 1_540_525_312 / 1_000_002,
 }
 
 
