@@ -385,11 +385,14 @@ int run_umma_passes(ic_cache* c, const ic_cache_plan_t& pl, const void* q_bf16, 
     const int v = atoi(env);
     if (v >= 0) up.seed_look_cycles = v;
   }
-  // CTAs of one partition may run an eighth of the partition's share of L2 apart (measured: with
-  // 18 partitions of 393 KB tiles, 3 tiles keep DRAM reads at the slab size, 8 tiles do not)
+  // CTAs of one partition may run half of the partition's share of L2 apart.  Progress is published
+  // at every PACE_EVERY-th tile only, so a word can be that stale (siblings in step still look
+  // PACE_EVERY apart) and a CTA moves on as many tiles between two looks: the window is what is left
+  // of the half share, and never less than the staleness plus some jitter.
   up.pace = pace;
   const int64_t tile_bytes = (int64_t)ROW_TILE * c->dim * 2;
-  up.pace_window = (int)std::max<int64_t>(2, std::min<int64_t>(16, (int64_t)c->l2_bytes / 8 / ((int64_t)P * tile_bytes)));
+  up.pace_window = (int)std::max<int64_t>(icc::PACE_EVERY + 2,
+      std::min<int64_t>(32, (int64_t)c->l2_bytes / 2 / ((int64_t)P * tile_bytes) - icc::PACE_EVERY));
   if (const char* env = getenv("IC_CACHE_PACE_WINDOW")) {   // tuning knob: tiles; 0 switches pacing off
     const int w = atoi(env);
     if (w <= 0) up.pace = nullptr;

@@ -84,6 +84,7 @@ cudaError_t scan_configure(int smem_optin);
 
 // tcgen05 scoring: query tiles of 128 (or one resident tile of 64) x row tiles of 256, top-k fused
 // in the epilogue.
+constexpr int PACE_EVERY = 4;   // a CTA publishes and compares its progress at every PACE_EVERY-th row tile
 struct UmmaParams {
   CUtensorMap tmap_q;     // [nq_pad, dim] bf16, box 64 x 128 (64 x 64 with q_resident), 128-byte swizzle
   CUtensorMap tmap_slab;  // [capacity, dim] bf16, box 64 x 256, 128-byte swizzle
@@ -104,7 +105,7 @@ struct UmmaParams {
   unsigned long long* pace;   // optional [n_part][units per partition] progress words (L2 pacing hint)
   unsigned epoch;             // number of this launch, unique in the process: tells this launch's progress
                               // words and seeding flags from older ones
-  int pace_window;            // tiles a CTA may run ahead of its slowest sibling
+  int pace_window;            // tiles a CTA may be ahead of the slowest published progress (>= PACE_EVERY + 2)
   float* seed_maxima;         // optional [n_query_tiles][n_part][seed_t0][128][4]: seeding inside the launch (needs
   unsigned* seed_flags;       // thr_floor == NULL and full first tiles); flags [n_query_tiles][n_part][4]
   int seed_look_cycles;       // longest an epilogue warp looks for its siblings' maxima, in SM cycles

@@ -124,7 +124,7 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* t
       : "memory");
 }
 // Same load issued by one CTA of a pair; the mbarrier may live in the peer CTA (address in
-// the cluster-wide shared window).  No multicast: each CTA fetches its own box.
+// the cluster-wide shared window).  Each CTA fetches its own box into its own shared memory.
 __device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorMap* tmap, int x, int y,
                                                  uint32_t bar_cluster_addr) {
   asm volatile(

@@ -265,9 +265,12 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       }
       // Pacing.  The CTAs (or pairs) that score different query tiles against the same
       // partition read the same row tiles; the tile comes from HBM once only while they stay
-      // within an L2-sized window of each other.  Each publishes how many tiles it has started
-      // and one that runs more than pace_window tiles ahead of the slowest holds its loads
-      // for a bounded time.  This is a bandwidth hint only: when the bound runs out it goes on.
+      // within an L2-sized window of each other.  They normally do by themselves (the ones behind
+      // find the tiles in L2 and catch up), so this is insurance against data-dependent drift and
+      // is kept cheap: only every PACE_EVERY-th tile a CTA publishes how many tiles it has started
+      // and looks at the others (a round trip to L2 that stalls this thread while the ring
+      // drains); one that is more than pace_window tiles ahead of the slowest word holds its
+      // loads for a bounded time.  A bandwidth hint only: when the bound runs out it goes on.
       const bool paced = (pace != nullptr) && units_per_part > 1 && rank == 0;
       volatile unsigned long long* pace_row = paced ? pace + (size_t)part * units_per_part : nullptr;
       const int my_unit = unit % units_per_part;
@@ -275,12 +278,13 @@ umma_score_topk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       constexpr int SUB = QRES ? 2 : 1;    // ring stages per K chunk of a row tile (resident: two halves of 128 rows)
       for (int64_t sq = 0; sq < n_seq && ok; ++sq, ++ordinal) {
         const int64_t tile = tile_of(sq);
-        if (paced) pace_row[my_unit] = ((unsigned long long)epoch << 32) | ordinal;
+        const bool look = paced && (ordinal % PACE_EVERY) == 0;
+        if (look) pace_row[my_unit] = ((unsigned long long)epoch << 32) | ordinal;
         for (int sub = 0; sub < SUB && ok; ++sub) {
           for (int kc = 0; kc < n_kc; ++kc, ++it) {
             ok = mbar_wait(&tail->empty[s], ph ^ 1u, abort_flag);
             if (!ok) break;
-            if (paced && kc == 0) {
+            if (look && kc == 0 && sub == 0) {
               const long long t0 = clock64();
               while (true) {
                 // all progress words are requested before the first is looked at (one round trip to
