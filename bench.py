@@ -48,12 +48,12 @@ NOMINAL_BF16_TFLOPS = 2250.0
 # rows scanned.  Key: (kernel, dim).  An entry is removed (the line then says null) whenever that
 # kernel changes after its capture.
 NCU_TRAFFIC_BYTES_PER_ROW = {
-    # profiles/umma_stress_2m_q1024.md: main pass, CTA pairs, 2,890,870,016 B over 1,877,632 scanned rows
-    ("umma_score_topk_kernel<2,streamed> (main pass)", 768): 2_890_870_016 / 1_877_632,
-    # profiles/umma_dense_1m_q256.md: CTA pairs, 2,095,134,464 B over 1,000,512 rows (incl. the re-read first tiles)
-    ("umma_score_topk_kernel<2,streamed> (main pass)", 1024): 2_095_134_464 / 1_000_512,
-    # profiles/umma_online_q64.md: resident query tile, 1,541,755,136 B over 1,000,128 rows
-    ("umma_score_topk_kernel<1,resident> (main pass)", 768): 1_541_755_136 / 1_000_128,
+    # profiles/umma_stress_2m_q1024.md: main pass, CTA pairs, 2,897,023,744 B over 1,877,632 scanned rows
+    ("umma_score_topk_kernel<2,streamed> (main pass)", 768): 2_897_023_744 / 1_877_632,
+    # profiles/umma_dense_1m_q256.md: CTA pairs, 2,095,586,048 B over 1,000,512 rows (incl. the re-read first tiles)
+    ("umma_score_topk_kernel<2,streamed> (main pass)", 1024): 2_095_586_048 / 1_000_512,
+    # profiles/umma_online_q64.md: resident query tile, 1,542,629,632 B over 1,000,128 rows
+    ("umma_score_topk_kernel<1,resident> (main pass)", 768): 1_542_629_632 / 1_000_128,
     # profiles/scan_online_q1.md: CUDA-core scan, 1,540,525,312 B over 1,000,002 rows
     ("scan_score_topk_kernel", 768): 1_540_525_312 / 1_000_002,
 }
