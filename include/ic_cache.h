@@ -94,9 +94,9 @@ typedef struct ic_cache_plan {
                             main pass, whose merged k-th key is the main pass's floor; the
                             main pass skips them (0 = none)                                */
   int32_t seed0_tiles;   /* tensor-core path: tiles (the first few of every partition, about
-                            one per SM in all) whose group maxima the CTAs of a launch
-                            exchange to agree on a first floor per query (0 = no seeding
-                            inside the launch)                                             */
+                            one per SM in all, more in a long sampling launch) whose group
+                            maxima the CTAs of a launch exchange to agree on a first floor
+                            per query (0 = no seeding inside the launch)                   */
   int32_t cta_group;     /* tensor-core path: 2 = CTA pairs issue one 256-query MMA and
                             split each row tile between them, 1 = single CTAs (else 0)     */
   int32_t query_resident;/* tensor-core path: 1 = at most 64 queries, M = 64, the whole query

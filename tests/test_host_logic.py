@@ -65,7 +65,8 @@ def test_plan_paths_and_shapes():
     assert p["n_query_tiles"] == 2 and p["n_partitions"] == 74 and p["n_ctas"] == 148
     p = pkg.ic_cache_plan(768, 16_000_000, 1024, 64)
     assert p["n_query_tiles"] == 8 and p["n_partitions"] == 18 and p["n_ctas"] == 144 and p["n_launches"] == 2
-    assert p["cta_group"] == 2 and p["seed0_tiles"] == 162 < p["seed_tiles"] and p["query_resident"] == 0   # 9 tiles for each of 18 partitions
+    # 24 tiles (a ninth of the sampling launch's 217 per CTA pair) for each of 18 partitions
+    assert p["cta_group"] == 2 and p["seed0_tiles"] == 432 < p["seed_tiles"] and p["query_resident"] == 0
     assert p["smem_bytes"] <= 232448
     assert p["seed_tiles"] > 0 and p["seed_tiles"] % 18 == 0 and p["seed_tiles"] * 256 * 15 < 16_000_000
     assert pkg.ic_cache_plan(768, 70_001, 64, 10)["seed_tiles"] == 0      # too few tiles per CTA
