@@ -48,8 +48,8 @@ NOMINAL_BF16_TFLOPS = 2250.0
 # rows scanned.  Key: (kernel, dim).  An entry is removed (the line then says null) whenever that
 # kernel changes after its capture.
 NCU_TRAFFIC_BYTES_PER_ROW = {
-    # profiles/umma_stress_2m_q1024.md: main pass, CTA pairs, 2,897,023,744 B over 1,877,632 scanned rows
-    ("umma_score_topk_kernel<2,streamed> (main pass)", 768): 2_897_023_744 / 1_877_632,
+    # profiles/umma_stress_2m_q1024.md: main pass, CTA pairs, 2,890,656,256 B over 1,877,632 scanned rows
+    ("umma_score_topk_kernel<2,streamed> (main pass)", 768): 2_890_656_256 / 1_877_632,
     # profiles/umma_dense_1m_q256.md: CTA pairs, 2,095,586,048 B over 1,000,512 rows (incl. the re-read first tiles)
     ("umma_score_topk_kernel<2,streamed> (main pass)", 1024): 2_095_586_048 / 1_000_512,
     # profiles/umma_online_q64.md: resident query tile, 1,542,629,632 B over 1,000,128 rows
