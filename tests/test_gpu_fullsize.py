@@ -94,6 +94,10 @@ def test_full_size_workloads_match_the_oracle_on_sampled_queries(loaded):
             # 16 M rows: one query of every 128-query tile (eight oracle queries for the batch of 1024)
             sample = sorted({min(nq - 1, t * 128 + (37 * t) % 128) for t in range((nq + 127) // 128)} | {0, nq - 1})
         loaded.check(nq, sample)
+    if w.n > 4_000_000:
+        # a batch size between the sweep's: two CTA pairs per row partition, and a sampling launch
+        # whose first floor comes from a different number of tiles per CTA
+        loaded.check(512, [t * 128 + (53 * t) % 128 for t in range(4)])
     if w.insert_rows:
         # streaming inserts between query batches; planted queries copy rows of the newest batch.
         # The oracle re-checks the first rounds and the last of the 20-round timed loop (round 19).
