@@ -119,6 +119,23 @@ def test_two_level_threshold_seeding(order):
     _seeding_case(order, 40, 16, 2_600_011, levels=2)
 
 
+@pytest.mark.parametrize("order", ["best_first", "best_last"])
+def test_long_sampling_launch_takes_its_first_floor_from_more_tiles(order):
+    """A batch of several query tiles against a cache large enough that the sampling launch runs
+    over dozens of tiles per CTA: it then exchanges the group maxima of more than the usual one
+    tile per SM.  The best rows sit all inside, or all outside, what is sampled."""
+    from paper_2501_12689_b200 import ic_cache_plan
+    dim, n, nq, k = 64, 12_000_517, 512, 10
+    plan = ic_cache_plan(dim, n, nq, k, IC_PATH_UMMA)
+    per_cta = plan["seed0_tiles"] // plan["n_partitions"]
+    assert plan["seed_tiles"] > 0 and plan["cta_group"] == 2 and per_cta > (148 + plan["n_partitions"] - 1) // plan["n_partitions"]
+    x, q = _gauss(n, dim, nq, seed=77)
+    s0 = (x.float() @ q[300].float())
+    x = x[torch.argsort(s0, descending=(order == "best_first"))].contiguous()
+    del s0
+    run_and_check(x, q, k, path=IC_PATH_UMMA, sample_queries=[0, 129, 300, 511], what=f"long sample/{order}")
+
+
 @pytest.mark.parametrize("nq,k", [(40, 10), (130, 64)])
 def test_seeding_falls_back_to_local_floors_when_the_siblings_are_not_waited_for(nq, k, monkeypatch):
     """The exchange of group maxima inside a launch is a bounded look, never a condition for
